@@ -1,0 +1,195 @@
+/*
+ * sablock.h -- C ABI of the B200 (sm_100a) implementation of SABlock's prefill-time
+ * KV-cache compression pass (semantic segmentation, observation-window scoring,
+ * segment-guided refinement, budget-driven adaptive block-size search, top-k selection
+ * and compaction of the retained K/V rows).
+ *
+ * Conventions (all entry points):
+ *  - "dev" pointers are CUDA device pointers owned by the caller; "host" pointers are
+ *    ordinary host memory.  The library never allocates or frees device memory: all
+ *    scratch comes from the caller's workspace `ws` (size from sablock_workspace_bytes).
+ *  - Device work is enqueued asynchronously on `stream` (a cudaStream_t passed as void*).
+ *    The return code reports host-side validation and launch errors only; on any error
+ *    nothing further is enqueued.  Conditions detected on the device (a bounded wait that
+ *    ran out, an internal consistency check) are written to a device status word that the
+ *    caller may read after synchronising (see sablock_read_status).
+ *  - Positions: a prompt has L tokens; the last W = `window` tokens are the observation
+ *    window and are never evicted; T = L - W is the compressible region (Sec. 3.1).
+ *  - Layouts: q_win [H, W, D]; k, v [L, Hkv, D] with element strides given in the
+ *    parameter block; all score vectors are fp32 of length T; indices are int32.
+ *  - `budget` counts every retained entry.  With budget_includes_window = 1 (default) the
+ *    W window entries are part of it, so Algorithm 2 runs with B = budget - W and exactly
+ *    `budget` rows are produced; with 0, B = budget and budget + W rows are produced.
+ *    If the rows to produce would be >= L the cache is returned unchanged (identity).
+ */
+#ifndef SABLOCK_H
+#define SABLOCK_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SABLOCK_OK = 0,
+    SABLOCK_ERR_INVALID_ARG = 1,
+    SABLOCK_ERR_UNSUPPORTED = 2,
+    SABLOCK_ERR_WORKSPACE_TOO_SMALL = 3,
+    SABLOCK_ERR_CUDA = 4,
+    SABLOCK_ERR_TIMEOUT = 5,
+    SABLOCK_ERR_INTERNAL = 6
+} sablock_status_t;
+
+typedef enum { SABLOCK_F32 = 0, SABLOCK_BF16 = 1 } sablock_dtype_t;
+
+/* Which kernel family computes the attention scores. AUTO picks the tensor-core
+ * (tcgen05) kernels whenever the shape allows it and the SIMT kernels otherwise. */
+typedef enum { SABLOCK_SCORE_AUTO = 0, SABLOCK_SCORE_SIMT = 1, SABLOCK_SCORE_TENSOR = 2 } sablock_score_impl_t;
+
+#define SABLOCK_MAX_SEQS 64        /* sequences per batched call              */
+#define SABLOCK_MAX_CANDIDATES 16  /* block-size candidates                   */
+
+typedef void *sablock_stream_t;    /* a cudaStream_t */
+
+/* Plain-data parameter block, passed by const pointer.  Fill it with
+ * sablock_params_default() and then set the shape fields. */
+typedef struct sablock_params {
+    int n_q_heads;                 /* H   query heads (Eq. 3 averages over these)               */
+    int n_kv_heads;                /* Hkv key/value heads; H % Hkv == 0 (grouped-query attention) */
+    int head_dim;                  /* D                                                         */
+    int window;                    /* W = n_rcnt, observation window (Sec. 3.1)                 */
+    int dtype;                     /* sablock_dtype_t of q_win, k, v, out_k, out_v              */
+    long long k_stride_token;      /* element strides of k; 0 = contiguous [L, Hkv, D]          */
+    long long k_stride_head;
+    long long k_stride_layer;      /* batched call only; 0 = total_tokens * k_stride_token      */
+    long long v_stride_token;      /* same for v                                                */
+    long long v_stride_head;
+    long long v_stride_layer;
+    float alpha;                   /* Eq. 8, default 0.9                                        */
+    float eta;                     /* Eq. 7, default 1.0                                        */
+    float eps;                     /* Eq. 6, default 1e-6                                       */
+    float tau;                     /* Eq. 12 fidelity threshold, default 0.85                   */
+    int pool_kernel;               /* 1 = no pooling (the paper's method); odd k > 1 pools s_t  */
+    int pool_mode;                 /* 0 = max, 1 = mean                                         */
+    int budget_includes_window;    /* default 1                                                 */
+    const unsigned *delim_bitmap;  /* dev: bit (id % 32) of word (id / 32) set <=> id delimits  */
+    int vocab_size;                /* ids outside [0, vocab_size) never delimit                 */
+    int score_impl;                /* sablock_score_impl_t                                      */
+    int l2_lag_tiles;              /* tuning knob of the tensor-core score kernel; 0 = default  */
+    int reserved[7];
+} sablock_params_t;
+
+void sablock_params_default(sablock_params_t *p);
+const char *sablock_status_string(sablock_status_t st);
+int sablock_version(void);
+size_t sablock_params_sizeof(void);   /* sizeof(sablock_params_t) as the library was built */
+
+/* Bytes of device scratch needed for a call over n_layers x n_seqs problems whose
+ * sequences have at most max_L tokens and total_tokens tokens in all.  Single-problem
+ * entry points use n_layers = n_seqs = 1, total_tokens = max_L = L.  Returns 0 on
+ * invalid arguments. */
+size_t sablock_workspace_bytes(const sablock_params_t *p, long long total_tokens, int max_L,
+                               int n_seqs, int n_layers);
+
+/* Where a fused call leaves its intermediate results inside the workspace, for diagnostics
+ * and tests: name is one of "s", "e", "s_refined" (f32 [n_layers][total_tokens], token row
+ * cu_seqlens[i] + t), "seg_id" (int32 [total_tokens]), "seg_start" (int32, sequence i at
+ * element cu_seqlens[i] + i), "n_seg" (int32 [n_seqs]).  Stores the byte offset and size;
+ * same arguments as sablock_workspace_bytes.  Returns SABLOCK_ERR_INVALID_ARG for an
+ * unknown name. */
+sablock_status_t sablock_workspace_region(const sablock_params_t *p, long long total_tokens, int max_L,
+                                          int n_seqs, int n_layers, const char *name,
+                                          size_t *offset, size_t *bytes);
+
+/* Reads (synchronously: it waits for `stream`) the device status word kept at the start of
+ * the workspace.  Returns SABLOCK_OK, SABLOCK_ERR_TIMEOUT or SABLOCK_ERR_INTERNAL; the raw
+ * word is stored to *raw (host) if not NULL. */
+sablock_status_t sablock_read_status(const void *ws, sablock_stream_t stream, int *raw);
+
+/* Stage 1 -- semantic segmentation (Sec. 3.1, "Semantic-Aware Segmentation").
+ * A token whose id is in the delimiter set is the last token of its segment.
+ *  token_ids dev int32[L]; seg_id dev int32[T] (segment index of each token);
+ *  seg_start dev int32[T+1] (first n_seg+1 entries valid, seg_start[n_seg] = T);
+ *  n_seg dev int32[1]. */
+sablock_status_t sablock_segment(const sablock_params_t *p, const int *token_ids, int L,
+                                 int *seg_id, int *seg_start, int *n_seg,
+                                 void *ws, size_t ws_bytes, sablock_stream_t stream);
+
+/* Stages 2+3 -- observation-window scoring (Sec. 3.2, Eqs. 2-4 and the per-token entropy of
+ * Eq. 6) followed by segment-guided refinement (Eqs. 5-8, Algorithm 1).
+ *  q_win dev [H, W, D]: queries of the last W prompt positions; k dev [L, Hkv, D];
+ *  seg_start / n_seg: from sablock_segment;
+ *  s dev f32[T] window score s_t (after pooling if enabled); e dev f32[T] or NULL: per-token
+ *  entropy; s_refined dev f32[T]; seg_stats dev f32[3*T] or NULL: I_k, D_k, omega_k in rows
+ *  of length T (first n_seg entries of each valid). */
+sablock_status_t sablock_score(const sablock_params_t *p, const void *q_win, const void *k, int L,
+                               const int *seg_start, const int *n_seg,
+                               float *s, float *e, float *s_refined, float *seg_stats,
+                               void *ws, size_t ws_bytes, sablock_stream_t stream);
+
+/* Stage 4 + index list -- Algorithm 2 (Sec. 3.3, Eqs. 9-13): global Top-B, implicit
+ * budgets, per-segment block-size search, aggregation.
+ *  block_candidates host int[n_candidates], strictly ascending, first entry 1;
+ *  out_idx dev int32[n_out]: retained positions, ascending, the W window positions last,
+ *  where n_out = budget (or budget + W, see budget_includes_window) or L for identity;
+ *  out_seg_block dev int32[T] or NULL: g*_k (0 where b_k = 0); out_seg_budget dev int32[T]
+ *  or NULL: b_k. */
+sablock_status_t sablock_select(const sablock_params_t *p, const float *s_refined, int L,
+                                const int *seg_start, const int *n_seg, int budget,
+                                const int *block_candidates, int n_candidates,
+                                int *out_idx, int *out_seg_block, int *out_seg_budget,
+                                void *ws, size_t ws_bytes, sablock_stream_t stream);
+
+/* Stage 5 -- merge with the recent tokens and compact (end of Sec. 3.3): copies rows
+ * out_idx[0..n_keep) of k and v into out_k, out_v dev [n_keep, Hkv, D] (contiguous). */
+sablock_status_t sablock_compact(const sablock_params_t *p, const void *k, const void *v, int L,
+                                 const int *out_idx, int n_keep, void *out_k, void *out_v,
+                                 sablock_stream_t stream);
+
+/* The whole pass for one layer of one sequence (Fig. 5 steps 1-4).
+ *  out_k, out_v dev [n_out, Hkv, D]; out_idx dev int32[n_out]; out_n_keep dev int32[1]. */
+sablock_status_t sablock_compress(const sablock_params_t *p, const void *q_win, const void *k,
+                                  const void *v, const int *token_ids, int L, int budget,
+                                  const int *block_candidates, int n_candidates,
+                                  void *out_k, void *out_v, int *out_idx, int *out_n_keep,
+                                  void *ws, size_t ws_bytes, sablock_stream_t stream);
+
+/* The whole pass for n_layers layers of n_seqs packed sequences in one launch sequence.
+ *  cu_seqlens host int[n_seqs+1], cu_seqlens[0] = 0: sequence i occupies packed token rows
+ *  [cu_seqlens[i], cu_seqlens[i+1]);
+ *  q_win dev [n_layers, n_seqs, H, W, D]; k, v dev [n_layers, total_tokens, Hkv, D] (strides
+ *  from the parameter block); token_ids dev int32[total_tokens] (shared by all layers);
+ *  out_k, out_v dev [n_layers, n_seqs, n_out, Hkv, D]; out_idx dev int32[n_layers, n_seqs,
+ *  n_out] (positions local to each sequence); out_n_keep dev int32[n_layers, n_seqs].
+ *  Sequences with L_i <= n_out are returned unchanged in their first L_i rows. */
+sablock_status_t sablock_compress_layers(const sablock_params_t *p, int n_layers, int n_seqs,
+                                         const void *q_win, const void *k, const void *v,
+                                         const int *token_ids, const int *cu_seqlens, int budget,
+                                         const int *block_candidates, int n_candidates,
+                                         void *out_k, void *out_v, int *out_idx, int *out_n_keep,
+                                         void *ws, size_t ws_bytes, sablock_stream_t stream);
+
+/* Same pass with HOST inputs and outputs (the end-to-end path): copies q_win, k, v and
+ * token_ids from host memory into the caller's device staging buffers (dev_*; same shapes
+ * as above), runs sablock_compress_layers, copies out_k, out_v, out_idx, out_n_keep back
+ * to host memory and waits for `stream`.  Pinned host memory makes the copies asynchronous
+ * with respect to each other; pageable memory also works. */
+sablock_status_t sablock_compress_layers_host(const sablock_params_t *p, int n_layers, int n_seqs,
+                                              const void *h_q_win, const void *h_k, const void *h_v,
+                                              const int *h_token_ids, const int *cu_seqlens, int budget,
+                                              const int *block_candidates, int n_candidates,
+                                              void *h_out_k, void *h_out_v, int *h_out_idx, int *h_out_n_keep,
+                                              void *dev_q_win, void *dev_k, void *dev_v, int *dev_token_ids,
+                                              void *dev_out_k, void *dev_out_v, int *dev_out_idx,
+                                              int *dev_out_n_keep,
+                                              void *ws, size_t ws_bytes, sablock_stream_t stream);
+
+/* Number of kernels the most recent entry-point call of this thread enqueued (for
+ * launch accounting in benchmarks). */
+int sablock_last_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SABLOCK_H */

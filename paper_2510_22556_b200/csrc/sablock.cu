@@ -1,0 +1,629 @@
+// C ABI of the SABlock compression library (see include/sablock.h): argument validation,
+// workspace planning, TMA tensor maps and kernel launches.  Every step of the pass runs in
+// the kernels of stages.cuh / score_simt.cuh / score_tc.cuh; there is no host fallback.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include "common.cuh"
+#include "stages.cuh"
+#include "score_simt.cuh"
+#include "score_tc.cuh"
+
+using namespace sab;
+
+namespace {
+
+thread_local int t_launches = 0;
+
+inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+
+struct Plan {
+    // geometry
+    Geo geo;
+    int n_prob, max_L;
+    bool use_tc;
+    int tpc1, tpc2;            // tiles per CTA of the tensor-core passes
+    int n_chunks;              // pass-1 partials per row
+    int keep_words, long_cap, seg_tiles;
+    // workspace offsets
+    size_t o_status, o_ticket, o_long_count, o_tile_state, o_keep, control_bytes;
+    size_t o_seg_id, o_seg_start, o_n_seg, o_s_raw, o_s, o_e, o_sr, o_part, o_lse, o_thr, o_cut, o_long_list,
+        o_phi, o_rank, total;
+};
+
+bool tc_eligible(const sablock_params_t* p)
+{
+    if (p->dtype != SABLOCK_BF16) return false;
+    if (p->head_dim != 64 && p->head_dim != 128) return false;
+    if (p->window != 8 && p->window != 16 && p->window != 32) return false;
+    const int G = p->n_q_heads / p->n_kv_heads;
+    if (G * p->window > 128) return false;
+    return true;
+}
+
+sablock_status_t validate_params(const sablock_params_t* p)
+{
+    if (!p) return SABLOCK_ERR_INVALID_ARG;
+    if (p->n_q_heads <= 0 || p->n_kv_heads <= 0 || p->n_q_heads % p->n_kv_heads) return SABLOCK_ERR_INVALID_ARG;
+    if (p->head_dim <= 0 || p->window <= 0) return SABLOCK_ERR_INVALID_ARG;
+    if (p->dtype != SABLOCK_F32 && p->dtype != SABLOCK_BF16) return SABLOCK_ERR_INVALID_ARG;
+    if (p->pool_kernel < 1 || (p->pool_kernel & 1) == 0) return SABLOCK_ERR_INVALID_ARG;
+    if (p->pool_mode != 0 && p->pool_mode != 1) return SABLOCK_ERR_INVALID_ARG;
+    if (p->score_impl < 0 || p->score_impl > 2) return SABLOCK_ERR_INVALID_ARG;
+    if (!(p->tau >= 0.f) || !(p->alpha >= 0.f) || !(p->eta >= 0.f) || !(p->eps >= 0.f)) return SABLOCK_ERR_INVALID_ARG;
+    if (p->k_stride_token < 0 || p->k_stride_head < 0 || p->k_stride_layer < 0 || p->v_stride_token < 0 ||
+        p->v_stride_head < 0 || p->v_stride_layer < 0)
+        return SABLOCK_ERR_INVALID_ARG;
+    if (p->window > kSimtMaxW || p->head_dim > kSimtMaxD) return SABLOCK_ERR_UNSUPPORTED;
+    if ((long long)p->n_q_heads * p->window > 2048) return SABLOCK_ERR_UNSUPPORTED;
+    const int es = p->dtype == SABLOCK_BF16 ? 2 : 4;
+    if ((p->head_dim * es) % 16) return SABLOCK_ERR_UNSUPPORTED;
+    if (p->score_impl == SABLOCK_SCORE_TENSOR && !tc_eligible(p)) return SABLOCK_ERR_UNSUPPORTED;
+    return SABLOCK_OK;
+}
+
+int elem_size(const sablock_params_t* p) { return p->dtype == SABLOCK_BF16 ? 2 : 4; }
+
+struct Strides { long long tok, head, layer; };
+Strides k_strides(const sablock_params_t* p, long long total_tokens)
+{
+    Strides s;
+    s.head = p->k_stride_head ? p->k_stride_head : p->head_dim;
+    s.tok = p->k_stride_token ? p->k_stride_token : (long long)p->n_kv_heads * p->head_dim;
+    s.layer = p->k_stride_layer ? p->k_stride_layer : total_tokens * s.tok;
+    return s;
+}
+Strides v_strides(const sablock_params_t* p, long long total_tokens)
+{
+    Strides s;
+    s.head = p->v_stride_head ? p->v_stride_head : p->head_dim;
+    s.tok = p->v_stride_token ? p->v_stride_token : (long long)p->n_kv_heads * p->head_dim;
+    s.layer = p->v_stride_layer ? p->v_stride_layer : total_tokens * s.tok;
+    return s;
+}
+
+// Builds geometry + workspace layout.  cu == NULL means one sequence of max_L tokens.
+sablock_status_t make_plan(const sablock_params_t* p, int n_layers, int n_seqs, const int* cu, long long total_tokens,
+                           int max_L, int n_out, Plan* pl)
+{
+    sablock_status_t st = validate_params(p);
+    if (st != SABLOCK_OK) return st;
+    if (n_layers < 1 || n_seqs < 1 || n_seqs > kMaxSeqs || max_L < 1 || total_tokens < max_L) return SABLOCK_ERR_INVALID_ARG;
+    if (total_tokens > 0x7fffffffLL || (long long)n_layers * total_tokens > (1LL << 40)) return SABLOCK_ERR_UNSUPPORTED;
+    memset(pl, 0, sizeof(*pl));
+    Geo& g = pl->geo;
+    g.n_layers = n_layers; g.n_seqs = n_seqs; g.total_tokens = (int)total_tokens; g.window = p->window;
+    g.H = p->n_q_heads; g.Hkv = p->n_kv_heads; g.D = p->head_dim; g.G = g.H / g.Hkv;
+    g.n_out = n_out; g.B = n_out - p->window;
+    if (cu) {
+        for (int i = 0; i <= n_seqs; ++i) g.cu[i] = cu[i];
+    } else {
+        g.cu[0] = 0; g.cu[1] = max_L;
+    }
+    pl->n_prob = n_layers * n_seqs;
+    pl->max_L = max_L;
+    // The TMA boxes are 128 rows tall: tensors with fewer rows go to the SIMT kernels.
+    const bool tc_rows_ok = total_tokens >= kTcTile && (long long)n_layers * n_seqs * g.H * g.window >= kTcTile;
+    pl->use_tc = p->score_impl == SABLOCK_SCORE_TENSOR ||
+                 (p->score_impl == SABLOCK_SCORE_AUTO && tc_eligible(p) && tc_rows_ok);
+    const long long tiles = (max_L + kTcTile - 1) / kTcTile;
+    if (pl->use_tc) {
+        long long work1 = tiles * g.Hkv * pl->n_prob, work2 = tiles * pl->n_prob;
+        pl->tpc1 = (int)fmin(8.0, fmax(1.0, (double)(work1 / (148 * 4))));
+        pl->tpc2 = (int)fmin(4.0, fmax(1.0, (double)(work2 / (148 * 4))));
+        pl->n_chunks = (int)((tiles + pl->tpc1 - 1) / pl->tpc1);
+    } else {
+        pl->tpc1 = pl->tpc2 = 1;
+        pl->n_chunks = (max_L + kSimtThreads - 1) / kSimtThreads;
+    }
+    pl->keep_words = (max_L + 31) / 32;
+    pl->long_cap = max_L / kSegShort + 1;
+    pl->seg_tiles = (max_L + kSegTile - 1) / kSegTile;
+
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes); return r; };
+    pl->o_status = take(64);
+    pl->o_ticket = take(sizeof(int) * n_seqs);
+    pl->o_long_count = take(sizeof(int) * pl->n_prob);
+    pl->o_tile_state = take(sizeof(unsigned long long) * (size_t)n_seqs * pl->seg_tiles);
+    pl->o_keep = take(sizeof(unsigned) * (size_t)pl->n_prob * pl->keep_words);
+    pl->control_bytes = o;
+    const size_t ntok = (size_t)n_layers * total_tokens;
+    pl->o_seg_id = take(sizeof(int) * total_tokens);
+    pl->o_seg_start = take(sizeof(int) * (total_tokens + n_seqs));
+    pl->o_n_seg = take(sizeof(int) * n_seqs);
+    pl->o_s_raw = take(p->pool_kernel > 1 ? sizeof(float) * ntok : 0);
+    pl->o_s = take(sizeof(float) * ntok);
+    pl->o_e = take(sizeof(float) * ntok);
+    pl->o_sr = take(sizeof(float) * ntok);
+    const size_t part_n = pl->use_tc ? (size_t)pl->n_prob * g.Hkv * pl->n_chunks * 128
+                                     : (size_t)pl->n_prob * g.H * g.window * pl->n_chunks;
+    pl->o_part = take(sizeof(float2) * part_n);
+    pl->o_lse = take(sizeof(float) * (size_t)pl->n_prob * g.H * g.window);
+    pl->o_thr = take(sizeof(unsigned) * pl->n_prob);
+    pl->o_cut = take(sizeof(int) * pl->n_prob);
+    pl->o_long_list = take(sizeof(int) * (size_t)pl->n_prob * pl->long_cap);
+    pl->o_phi = take(sizeof(double) * ntok);
+    pl->o_rank = take(sizeof(int) * ntok);
+    pl->total = o;
+    return SABLOCK_OK;
+}
+
+template <typename T> T* at(void* ws, size_t off) { return reinterpret_cast<T*>(static_cast<char*>(ws) + off); }
+
+sablock_status_t check_launch()
+{
+    ++t_launches;
+    return cudaGetLastError() == cudaSuccess ? SABLOCK_OK : SABLOCK_ERR_CUDA;
+}
+#define SAB_TRY(expr) do { sablock_status_t _s = (expr); if (_s != SABLOCK_OK) return _s; } while (0)
+
+sablock_status_t zero_control(const Plan& pl, void* ws, cudaStream_t stream)
+{
+    return cudaMemsetAsync(ws, 0, pl.control_bytes, stream) == cudaSuccess ? SABLOCK_OK : SABLOCK_ERR_CUDA;
+}
+
+// ------------------------------------------------------------------ stage launchers
+sablock_status_t run_segment(const Plan& pl, const sablock_params_t* p, const int* token_ids, int* seg_id,
+                             int* seg_start, int* n_seg, void* ws, cudaStream_t stream)
+{
+    if (!token_ids || !seg_id || !seg_start || !n_seg || !p->delim_bitmap || p->vocab_size <= 0)
+        return SABLOCK_ERR_INVALID_ARG;
+    dim3 grid(pl.seg_tiles, pl.geo.n_seqs);
+    segment_kernel<<<grid, kSegThreads, 0, stream>>>(pl.geo, token_ids, p->delim_bitmap, p->vocab_size, seg_id,
+                                                     seg_start, n_seg, at<unsigned long long>(ws, pl.o_tile_state),
+                                                     at<int>(ws, pl.o_ticket), pl.seg_tiles, at<int>(ws, pl.o_status));
+    return check_launch();
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+sablock_status_t make_tensor_maps(const Plan& pl, const sablock_params_t* p, const void* q, const void* k,
+                                  CUtensorMap* tmQ, CUtensorMap* tmK)
+{
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return SABLOCK_ERR_CUDA;
+    const Geo& g = pl.geo;
+    const Strides ks = k_strides(p, g.total_tokens);
+    if (g.total_tokens < kTcTile || (long long)pl.n_prob * g.H * g.window < kTcTile) return SABLOCK_ERR_UNSUPPORTED;
+    if ((reinterpret_cast<uintptr_t>(q) & 15) || (reinterpret_cast<uintptr_t>(k) & 15) || (ks.head * 2) % 16 ||
+        (ks.tok * 2) % 16 || (ks.layer * 2) % 16)
+        return SABLOCK_ERR_UNSUPPORTED;
+    {   // queries as rows: [n_prob * H * W, D]
+        cuuint64_t dims[2] = {(cuuint64_t)g.D, (cuuint64_t)pl.n_prob * g.H * g.window};
+        cuuint64_t strides[1] = {(cuuint64_t)g.D * 2};
+        cuuint32_t box[2] = {64, 128};
+        cuuint32_t estr[2] = {1, 1};
+        if (enc(tmQ, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(q), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return SABLOCK_ERR_CUDA;
+    }
+    {   // keys: [layer][token][kv head][D]
+        cuuint64_t dims[4] = {(cuuint64_t)g.D, (cuuint64_t)g.Hkv, (cuuint64_t)g.total_tokens, (cuuint64_t)g.n_layers};
+        cuuint64_t strides[3] = {(cuuint64_t)ks.head * 2, (cuuint64_t)ks.tok * 2, (cuuint64_t)ks.layer * 2};
+        cuuint32_t box[4] = {64, 1, 128, 1};
+        cuuint32_t estr[4] = {1, 1, 1, 1};
+        if (enc(tmK, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(k), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return SABLOCK_ERR_CUDA;
+    }
+    return SABLOCK_OK;
+}
+
+template <int W>
+sablock_status_t launch_p2_tc(const Plan& pl, const CUtensorMap& tmQ, const CUtensorMap& tmK, float c2, float eps,
+                              ScoreBufs sb, float* s, float* e, int* status, cudaStream_t stream)
+{
+    constexpr int NST = 3;
+    const int n_atoms = pl.geo.D / 64;
+    const int smem = 1024 + NST * 2 * n_atoms * kAtomBytes;
+    auto kern = score_p2_tc<W, NST>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+        return SABLOCK_ERR_CUDA;
+    const int tiles = (pl.max_L + kTcTile - 1) / kTcTile;
+    dim3 grid((tiles + pl.tpc2 - 1) / pl.tpc2, pl.n_prob);
+    kern<<<grid, kTcThreads, smem, stream>>>(tmQ, tmK, pl.geo, c2, eps, sb, pl.tpc2, s, e, status);
+    return check_launch();
+}
+
+// Stage 2: window scores s (pre-pooling) and per-token entropy e.
+sablock_status_t run_score(const Plan& pl, const sablock_params_t* p, const void* q, const void* k, float* s,
+                           float* e, void* ws, cudaStream_t stream)
+{
+    if (!q || !k || !s || !e) return SABLOCK_ERR_INVALID_ARG;
+    const Geo& g = pl.geo;
+    const float c2 = (float)(1.4426950408889634 / sqrt((double)g.D));
+    ScoreBufs sb;
+    sb.part = at<float2>(ws, pl.o_part);
+    sb.lse2 = at<float>(ws, pl.o_lse);
+    sb.n_chunks = pl.n_chunks;
+    int* status = at<int>(ws, pl.o_status);
+    const Strides ks = k_strides(p, g.total_tokens);
+    if (pl.use_tc) {
+        CUtensorMap tmQ, tmK;
+        SAB_TRY(make_tensor_maps(pl, p, q, k, &tmQ, &tmK));
+        constexpr int NST1 = 2;
+        const int n_atoms = g.D / 64;
+        const int smem1 = 1024 + (1 + NST1) * n_atoms * kAtomBytes;
+        auto k1 = score_p1_tc<NST1>;
+        if (cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, smem1) != cudaSuccess)
+            return SABLOCK_ERR_CUDA;
+        dim3 grid1(pl.n_chunks, g.Hkv, pl.n_prob);
+        k1<<<grid1, kTcThreads, smem1, stream>>>(tmQ, tmK, g, c2, sb, pl.tpc1, status);
+        SAB_TRY(check_launch());
+        lse_merge_tc<<<dim3(g.Hkv, pl.n_prob), 128, 0, stream>>>(g, sb, pl.tpc1);
+        SAB_TRY(check_launch());
+        switch (g.window) {
+            case 8: return launch_p2_tc<8>(pl, tmQ, tmK, c2, p->eps, sb, s, e, status, stream);
+            case 16: return launch_p2_tc<16>(pl, tmQ, tmK, c2, p->eps, sb, s, e, status, stream);
+            case 32: return launch_p2_tc<32>(pl, tmQ, tmK, c2, p->eps, sb, s, e, status, stream);
+            default: return SABLOCK_ERR_UNSUPPORTED;
+        }
+    }
+    const int smem1 = (g.window * g.D + 2 * (kSimtThreads / 32) * g.window) * (int)sizeof(float);
+    const int smem2 = (kSimtWChunk * g.D + kSimtWChunk) * (int)sizeof(float);
+    dim3 grid1(pl.n_chunks, g.H, pl.n_prob);
+    dim3 grid2((pl.max_L + kSimtThreads - 1) / kSimtThreads, pl.n_prob);
+    dim3 gridm((g.H * g.window + 127) / 128, pl.n_prob);
+    if (p->dtype == SABLOCK_BF16) {
+        auto k1 = score_p1_simt<__nv_bfloat16>;
+        if (cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, smem1) != cudaSuccess)
+            return SABLOCK_ERR_CUDA;
+        k1<<<grid1, kSimtThreads, smem1, stream>>>(g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, ks.tok, ks.head,
+                                                   ks.layer, c2, sb);
+        SAB_TRY(check_launch());
+        lse_merge_simt<<<gridm, 128, 0, stream>>>(g, sb);
+        SAB_TRY(check_launch());
+        score_p2_simt<__nv_bfloat16><<<grid2, kSimtThreads, smem2, stream>>>(
+            g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, ks.tok, ks.head, ks.layer, c2, p->eps, sb, s, e);
+    } else {
+        auto k1 = score_p1_simt<float>;
+        if (cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, smem1) != cudaSuccess)
+            return SABLOCK_ERR_CUDA;
+        k1<<<grid1, kSimtThreads, smem1, stream>>>(g, (const float*)q, (const float*)k, ks.tok, ks.head, ks.layer, c2, sb);
+        SAB_TRY(check_launch());
+        lse_merge_simt<<<gridm, 128, 0, stream>>>(g, sb);
+        SAB_TRY(check_launch());
+        score_p2_simt<float><<<grid2, kSimtThreads, smem2, stream>>>(g, (const float*)q, (const float*)k, ks.tok,
+                                                                     ks.head, ks.layer, c2, p->eps, sb, s, e);
+    }
+    return check_launch();
+}
+
+// Stage 3 (with optional pooling first): s_raw -> s (pooled) -> s_refined.
+sablock_status_t run_refine(const Plan& pl, const sablock_params_t* p, const float* s_raw, float* s, const float* e,
+                            const int* seg_start, const int* n_seg, float* s_ref, float* stats, int stats_stride,
+                            cudaStream_t stream)
+{
+    const int gx = (int)fmin(32.0, fmax(1.0, (double)((pl.max_L + 2047) / 2048)));
+    if (p->pool_kernel > 1) {
+        pool_kernel<<<dim3(gx * 4, pl.n_prob), 256, 0, stream>>>(pl.geo, s_raw, s, p->pool_kernel, p->pool_mode);
+        SAB_TRY(check_launch());
+    }
+    refine_kernel<<<dim3(gx, pl.n_prob), 256, 0, stream>>>(pl.geo, s, e, seg_start, n_seg, p->alpha, p->eta, s_ref,
+                                                           stats, stats_stride);
+    return check_launch();
+}
+
+sablock_status_t check_candidates(const int* cand, int n, Cands* out)
+{
+    if (!cand || n < 1 || n > kMaxCand || cand[0] != 1) return SABLOCK_ERR_INVALID_ARG;
+    for (int i = 1; i < n; ++i)
+        if (cand[i] <= cand[i - 1]) return SABLOCK_ERR_INVALID_ARG;
+    out->n = n;
+    for (int i = 0; i < n; ++i) out->g[i] = cand[i];
+    return SABLOCK_OK;
+}
+
+// Stage 4 + index list.
+sablock_status_t run_select(const Plan& pl, const sablock_params_t* p, const float* s_ref, const int* seg_start,
+                            const int* n_seg, const Cands& cands, int* out_idx, int* out_n_keep, int* seg_g,
+                            int* seg_b, int seg_stride, void* ws, cudaStream_t stream)
+{
+    const Geo& g = pl.geo;
+    unsigned* thr = at<unsigned>(ws, pl.o_thr);
+    int* cut = at<int>(ws, pl.o_cut);
+    topb_kernel<<<pl.n_prob, kTopThreads, 0, stream>>>(g, s_ref, thr, cut);
+    SAB_TRY(check_launch());
+    SearchOut so;
+    so.keep = at<unsigned>(ws, pl.o_keep);
+    so.keep_words = pl.keep_words;
+    so.seg_g = seg_g; so.seg_b = seg_b; so.seg_stride = seg_stride;
+    so.long_list = at<int>(ws, pl.o_long_list);
+    so.long_count = at<int>(ws, pl.o_long_count);
+    so.long_cap = pl.long_cap;
+    const int gx = (int)fmin(32.0, fmax(1.0, (double)((pl.max_L + 2047) / 2048)));
+    search_kernel<<<dim3(gx, pl.n_prob), kSearchWarps * 32, 0, stream>>>(g, cands, s_ref, seg_start, n_seg, thr, cut,
+                                                                        p->tau, so);
+    SAB_TRY(check_launch());
+    search_long_kernel<<<dim3(4, pl.n_prob), kLongThreads, 0, stream>>>(g, cands, s_ref, seg_start, thr, cut, p->tau, so,
+                                                                       at<double>(ws, pl.o_phi), at<int>(ws, pl.o_rank));
+    SAB_TRY(check_launch());
+    index_kernel<<<pl.n_prob, kIdxThreads, 0, stream>>>(g, so.keep, pl.keep_words, out_idx, out_n_keep,
+                                                        at<int>(ws, pl.o_status));
+    return check_launch();
+}
+
+sablock_status_t run_compact(const Geo& g, int n_prob, const sablock_params_t* p, const void* k, const void* v,
+                             const int* out_idx, const int* out_n_keep, int n_keep_fixed, void* out_k, void* out_v,
+                             cudaStream_t stream)
+{
+    if (!k || !v || !out_idx || !out_k || !out_v) return SABLOCK_ERR_INVALID_ARG;
+    const int es = elem_size(p);
+    const Strides ks = k_strides(p, g.total_tokens), vs = v_strides(p, g.total_tokens);
+    CompactArgs c;
+    c.k = (const char*)k; c.v = (const char*)v; c.out_k = (char*)out_k; c.out_v = (char*)out_v;
+    c.k_tok = ks.tok * es; c.k_head = ks.head * es; c.k_layer = ks.layer * es;
+    c.v_tok = vs.tok * es; c.v_head = vs.head * es; c.v_layer = vs.layer * es;
+    c.head_bytes = g.D * es;
+    c.rows_per_cta = 4;
+    const long long all[] = {c.k_tok, c.k_head, c.k_layer, c.v_tok, c.v_head, c.v_layer};
+    for (long long x : all)
+        if (x % 16) return SABLOCK_ERR_UNSUPPORTED;
+    if ((reinterpret_cast<uintptr_t>(k) | reinterpret_cast<uintptr_t>(v) | reinterpret_cast<uintptr_t>(out_k) |
+         reinterpret_cast<uintptr_t>(out_v)) & 15)
+        return SABLOCK_ERR_UNSUPPORTED;
+    dim3 grid((g.n_out + c.rows_per_cta - 1) / c.rows_per_cta, n_prob, 2);
+    compact_kernel<<<grid, 256, 0, stream>>>(g, c, out_idx, out_n_keep, n_keep_fixed);
+    return check_launch();
+}
+
+int rows_out(const sablock_params_t* p, int budget) { return p->budget_includes_window ? budget : budget + p->window; }
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------
+// C ABI
+// ---------------------------------------------------------------------------------------
+extern "C" {
+
+void sablock_params_default(sablock_params_t* p)
+{
+    if (!p) return;
+    memset(p, 0, sizeof(*p));
+    p->dtype = SABLOCK_BF16;
+    p->alpha = 0.9f; p->eta = 1.0f; p->eps = 1e-6f; p->tau = 0.85f;     // Sec. 4.1, implementation details
+    p->pool_kernel = 1; p->pool_mode = 0;
+    p->budget_includes_window = 1;
+    p->score_impl = SABLOCK_SCORE_AUTO;
+}
+
+const char* sablock_status_string(sablock_status_t st)
+{
+    switch (st) {
+        case SABLOCK_OK: return "ok";
+        case SABLOCK_ERR_INVALID_ARG: return "invalid argument";
+        case SABLOCK_ERR_UNSUPPORTED: return "unsupported shape, dtype or alignment";
+        case SABLOCK_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case SABLOCK_ERR_CUDA: return "CUDA runtime or driver error";
+        case SABLOCK_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+        case SABLOCK_ERR_INTERNAL: return "internal consistency check failed on the device";
+    }
+    return "unknown status";
+}
+
+int sablock_version(void) { return 100; }
+
+size_t sablock_params_sizeof(void) { return sizeof(sablock_params_t); }
+
+int sablock_last_launch_count(void) { return t_launches; }
+
+size_t sablock_workspace_bytes(const sablock_params_t* p, long long total_tokens, int max_L, int n_seqs, int n_layers)
+{
+    Plan pl;
+    if (n_seqs < 1 || n_seqs > kMaxSeqs) return 0;
+    int cu[kMaxSeqs + 1];
+    // Offsets depend on totals only, not on where the sequence boundaries fall.
+    for (int i = 0; i <= n_seqs; ++i) cu[i] = 0;
+    cu[n_seqs] = (int)total_tokens;
+    if (make_plan(p, n_layers, n_seqs, cu, total_tokens, max_L, p ? p->window + 1 : 1, &pl) != SABLOCK_OK) return 0;
+    return pl.total;
+}
+
+sablock_status_t sablock_workspace_region(const sablock_params_t* p, long long total_tokens, int max_L, int n_seqs,
+                                          int n_layers, const char* name, size_t* offset, size_t* bytes)
+{
+    if (!name || !offset || !bytes || n_seqs < 1 || n_seqs > kMaxSeqs) return SABLOCK_ERR_INVALID_ARG;
+    Plan pl;
+    int cu[kMaxSeqs + 1];
+    for (int i = 0; i <= n_seqs; ++i) cu[i] = 0;
+    cu[n_seqs] = (int)total_tokens;
+    SAB_TRY(make_plan(p, n_layers, n_seqs, cu, total_tokens, max_L, p->window + 1, &pl));
+    const size_t ntok = (size_t)n_layers * total_tokens;
+    struct { const char* n; size_t off, sz; } tab[] = {
+        {"s", pl.o_s, sizeof(float) * ntok},           {"e", pl.o_e, sizeof(float) * ntok},
+        {"s_refined", pl.o_sr, sizeof(float) * ntok},  {"seg_id", pl.o_seg_id, sizeof(int) * (size_t)total_tokens},
+        {"seg_start", pl.o_seg_start, sizeof(int) * (size_t)(total_tokens + n_seqs)},
+        {"n_seg", pl.o_n_seg, sizeof(int) * (size_t)n_seqs},
+    };
+    for (auto& t : tab)
+        if (!strcmp(t.n, name)) { *offset = t.off; *bytes = t.sz; return SABLOCK_OK; }
+    return SABLOCK_ERR_INVALID_ARG;
+}
+
+sablock_status_t sablock_read_status(const void* ws, sablock_stream_t stream, int* raw)
+{
+    if (!ws) return SABLOCK_ERR_INVALID_ARG;
+    int word = 0;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(&word, ws, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return SABLOCK_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return SABLOCK_ERR_CUDA;
+    if (raw) *raw = word;
+    if (word & kStatTimeout) return SABLOCK_ERR_TIMEOUT;
+    if (word & kStatInternal) return SABLOCK_ERR_INTERNAL;
+    return SABLOCK_OK;
+}
+
+sablock_status_t sablock_segment(const sablock_params_t* p, const int* token_ids, int L, int* seg_id, int* seg_start,
+                                 int* n_seg, void* ws, size_t ws_bytes, sablock_stream_t stream)
+{
+    t_launches = 0;
+    if (!p || L <= p->window) return SABLOCK_ERR_INVALID_ARG;
+    Plan pl;
+    SAB_TRY(make_plan(p, 1, 1, nullptr, L, L, p->window + 1, &pl));
+    if (!ws || ws_bytes < pl.total) return SABLOCK_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    SAB_TRY(zero_control(pl, ws, st));
+    return run_segment(pl, p, token_ids, seg_id, seg_start, n_seg, ws, st);
+}
+
+sablock_status_t sablock_score(const sablock_params_t* p, const void* q_win, const void* k, int L, const int* seg_start,
+                               const int* n_seg, float* s, float* e, float* s_refined, float* seg_stats, void* ws,
+                               size_t ws_bytes, sablock_stream_t stream)
+{
+    t_launches = 0;
+    if (!p || L <= p->window || !seg_start || !n_seg || !s || !s_refined) return SABLOCK_ERR_INVALID_ARG;
+    Plan pl;
+    SAB_TRY(make_plan(p, 1, 1, nullptr, L, L, p->window + 1, &pl));
+    if (!ws || ws_bytes < pl.total) return SABLOCK_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    SAB_TRY(zero_control(pl, ws, st));
+    float* e_buf = e ? e : at<float>(ws, pl.o_e);
+    float* s_raw = p->pool_kernel > 1 ? at<float>(ws, pl.o_s_raw) : s;
+    SAB_TRY(run_score(pl, p, q_win, k, s_raw, e_buf, ws, st));
+    return run_refine(pl, p, s_raw, s, e_buf, seg_start, n_seg, s_refined, seg_stats, L - p->window, st);
+}
+
+sablock_status_t sablock_select(const sablock_params_t* p, const float* s_refined, int L, const int* seg_start,
+                                const int* n_seg, int budget, const int* block_candidates, int n_candidates,
+                                int* out_idx, int* out_seg_block, int* out_seg_budget, void* ws, size_t ws_bytes,
+                                sablock_stream_t stream)
+{
+    t_launches = 0;
+    if (!p || L < 1 || !s_refined || !seg_start || !n_seg || !out_idx) return SABLOCK_ERR_INVALID_ARG;
+    if (budget <= (p->budget_includes_window ? p->window : 0)) return SABLOCK_ERR_INVALID_ARG;
+    Cands cands;
+    SAB_TRY(check_candidates(block_candidates, n_candidates, &cands));
+    Plan pl;
+    SAB_TRY(make_plan(p, 1, 1, nullptr, L, L, rows_out(p, budget), &pl));
+    if (!ws || ws_bytes < pl.total) return SABLOCK_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    SAB_TRY(zero_control(pl, ws, st));
+    // the retained count is written to workspace (n_seg slot is free here)
+    return run_select(pl, p, s_refined, seg_start, n_seg, cands, out_idx, at<int>(ws, pl.o_n_seg), out_seg_block,
+                      out_seg_budget, L > p->window ? L - p->window : 1, ws, st);
+}
+
+sablock_status_t sablock_compact(const sablock_params_t* p, const void* k, const void* v, int L, const int* out_idx,
+                                 int n_keep, void* out_k, void* out_v, sablock_stream_t stream)
+{
+    t_launches = 0;
+    if (!p || L < 1 || n_keep < 1 || n_keep > L) return SABLOCK_ERR_INVALID_ARG;
+    SAB_TRY(validate_params(p));
+    Geo g;
+    memset(&g, 0, sizeof(g));
+    g.n_layers = g.n_seqs = 1; g.total_tokens = L; g.window = p->window;
+    g.H = p->n_q_heads; g.Hkv = p->n_kv_heads; g.D = p->head_dim; g.G = g.H / g.Hkv;
+    g.n_out = n_keep; g.B = n_keep - p->window;
+    g.cu[0] = 0; g.cu[1] = L;
+    return run_compact(g, 1, p, k, v, out_idx, nullptr, n_keep, out_k, out_v, static_cast<cudaStream_t>(stream));
+}
+
+sablock_status_t sablock_compress_layers(const sablock_params_t* p, int n_layers, int n_seqs, const void* q_win,
+                                         const void* k, const void* v, const int* token_ids, const int* cu_seqlens,
+                                         int budget, const int* block_candidates, int n_candidates, void* out_k,
+                                         void* out_v, int* out_idx, int* out_n_keep, void* ws, size_t ws_bytes,
+                                         sablock_stream_t stream)
+{
+    t_launches = 0;
+    if (!p || !cu_seqlens || n_seqs < 1 || n_seqs > kMaxSeqs || n_layers < 1) return SABLOCK_ERR_INVALID_ARG;
+    if (!q_win || !k || !v || !token_ids || !out_k || !out_v || !out_idx || !out_n_keep) return SABLOCK_ERR_INVALID_ARG;
+    if (budget <= (p->budget_includes_window ? p->window : 0)) return SABLOCK_ERR_INVALID_ARG;
+    if (cu_seqlens[0] != 0) return SABLOCK_ERR_INVALID_ARG;
+    int max_L = 0;
+    for (int i = 0; i < n_seqs; ++i) {
+        const int L = cu_seqlens[i + 1] - cu_seqlens[i];
+        if (L < 1) return SABLOCK_ERR_INVALID_ARG;
+        if (L > max_L) max_L = L;
+    }
+    Cands cands;
+    SAB_TRY(check_candidates(block_candidates, n_candidates, &cands));
+    Plan pl;
+    SAB_TRY(make_plan(p, n_layers, n_seqs, cu_seqlens, cu_seqlens[n_seqs], max_L, rows_out(p, budget), &pl));
+    if (!ws || ws_bytes < pl.total) return SABLOCK_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    SAB_TRY(zero_control(pl, ws, st));
+    int* seg_id = at<int>(ws, pl.o_seg_id);
+    int* seg_start = at<int>(ws, pl.o_seg_start);
+    int* n_seg = at<int>(ws, pl.o_n_seg);
+    float* s = at<float>(ws, pl.o_s);
+    float* e = at<float>(ws, pl.o_e);
+    float* sr = at<float>(ws, pl.o_sr);
+    float* s_raw = p->pool_kernel > 1 ? at<float>(ws, pl.o_s_raw) : s;
+    SAB_TRY(run_segment(pl, p, token_ids, seg_id, seg_start, n_seg, ws, st));
+    SAB_TRY(run_score(pl, p, q_win, k, s_raw, e, ws, st));
+    SAB_TRY(run_refine(pl, p, s_raw, s, e, seg_start, n_seg, sr, nullptr, 0, st));
+    SAB_TRY(run_select(pl, p, sr, seg_start, n_seg, cands, out_idx, out_n_keep, nullptr, nullptr, 0, ws, st));
+    return run_compact(pl.geo, pl.n_prob, p, k, v, out_idx, out_n_keep, 0, out_k, out_v, st);
+}
+
+sablock_status_t sablock_compress(const sablock_params_t* p, const void* q_win, const void* k, const void* v,
+                                  const int* token_ids, int L, int budget, const int* block_candidates,
+                                  int n_candidates, void* out_k, void* out_v, int* out_idx, int* out_n_keep, void* ws,
+                                  size_t ws_bytes, sablock_stream_t stream)
+{
+    if (L < 1) return SABLOCK_ERR_INVALID_ARG;
+    const int cu[2] = {0, L};
+    return sablock_compress_layers(p, 1, 1, q_win, k, v, token_ids, cu, budget, block_candidates, n_candidates, out_k,
+                                   out_v, out_idx, out_n_keep, ws, ws_bytes, stream);
+}
+
+sablock_status_t sablock_compress_layers_host(const sablock_params_t* p, int n_layers, int n_seqs, const void* h_q_win,
+                                              const void* h_k, const void* h_v, const int* h_token_ids,
+                                              const int* cu_seqlens, int budget, const int* block_candidates,
+                                              int n_candidates, void* h_out_k, void* h_out_v, int* h_out_idx,
+                                              int* h_out_n_keep, void* dev_q_win, void* dev_k, void* dev_v,
+                                              int* dev_token_ids, void* dev_out_k, void* dev_out_v, int* dev_out_idx,
+                                              int* dev_out_n_keep, void* ws, size_t ws_bytes, sablock_stream_t stream)
+{
+    if (!p || !cu_seqlens || n_seqs < 1 || n_seqs > kMaxSeqs || n_layers < 1) return SABLOCK_ERR_INVALID_ARG;
+    if (!h_q_win || !h_k || !h_v || !h_token_ids || !h_out_k || !h_out_v || !h_out_idx || !h_out_n_keep ||
+        !dev_q_win || !dev_k || !dev_v || !dev_token_ids)
+        return SABLOCK_ERR_INVALID_ARG;
+    if (p->k_stride_token || p->k_stride_head || p->k_stride_layer || p->v_stride_token || p->v_stride_head ||
+        p->v_stride_layer)
+        return SABLOCK_ERR_UNSUPPORTED;            // host staging assumes contiguous tensors
+    SAB_TRY(validate_params(p));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t es = elem_size(p);
+    const size_t total = (size_t)cu_seqlens[n_seqs];
+    const size_t kv_bytes = (size_t)n_layers * total * p->n_kv_heads * p->head_dim * es;
+    const size_t q_bytes = (size_t)n_layers * n_seqs * p->n_q_heads * p->window * p->head_dim * es;
+    const int n_out = rows_out(p, budget);
+    const size_t n_prob = (size_t)n_layers * n_seqs;
+    const size_t okv_bytes = n_prob * n_out * p->n_kv_heads * p->head_dim * es;
+    if (cudaMemcpyAsync(dev_token_ids, h_token_ids, total * sizeof(int), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(dev_q_win, h_q_win, q_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(dev_k, h_k, kv_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(dev_v, h_v, kv_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return SABLOCK_ERR_CUDA;
+    SAB_TRY(sablock_compress_layers(p, n_layers, n_seqs, dev_q_win, dev_k, dev_v, dev_token_ids, cu_seqlens, budget,
+                                    block_candidates, n_candidates, dev_out_k, dev_out_v, dev_out_idx, dev_out_n_keep,
+                                    ws, ws_bytes, stream));
+    if (cudaMemcpyAsync(h_out_k, dev_out_k, okv_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaMemcpyAsync(h_out_v, dev_out_v, okv_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaMemcpyAsync(h_out_idx, dev_out_idx, n_prob * n_out * sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaMemcpyAsync(h_out_n_keep, dev_out_n_keep, n_prob * sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return SABLOCK_ERR_CUDA;
+    return cudaStreamSynchronize(st) == cudaSuccess ? SABLOCK_OK : SABLOCK_ERR_CUDA;
+}
+
+}  // extern "C"

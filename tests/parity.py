@@ -1,0 +1,81 @@
+"""GPU-vs-oracle comparison protocol shared by the GPU tests, the smoke check and the bench.
+
+Scores: |gpu - ref| <= ABS + REL * |ref| with the tolerance the benchmark spec states for bf16 inputs
+with fp32 accumulation (rel 2e-3, abs 1e-5).  Integer results (segment ids, indices, block
+sizes) and K/V bytes: bit-exact.  Where the oracle's float64 scores make a decision on a gap
+smaller than the score tolerance, the index comparison is tie-aware: Algorithm 2 is re-run
+by the oracle on the GPU's own fp32 refined scores and must reproduce the GPU's indices
+exactly.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import oracle
+
+REL, ABS = 2e-3, 1e-5
+
+
+def assert_scores_close(gpu: torch.Tensor, ref: np.ndarray, what: str, rel: float = REL, abs_: float = ABS):
+    g = gpu.detach().cpu().double().numpy()
+    assert g.shape == ref.shape, (what, g.shape, ref.shape)
+    assert np.isfinite(g).all(), f"{what}: non-finite values"
+    err = np.abs(g - ref)
+    bound = abs_ + rel * np.abs(ref)
+    bad = err > bound
+    if bad.any():
+        i = int(np.argmax(err - bound))
+        raise AssertionError(f"{what}: {int(bad.sum())} of {g.size} outside tolerance; worst at {i}: "
+                             f"gpu={g[i]:.9g} ref={ref[i]:.9g}")
+    denom = np.maximum(np.abs(ref), 1e-30)
+    return float((err / denom).max())
+
+
+def check_problem(cfg_like, q, k, v, ids, bitmap, vocab, budget, candidates, out_k, out_v, out_idx, n_keep,
+                  s_gpu=None, e_gpu=None, sr_gpu=None, params=None, strict_scores=True):
+    """Full protocol for one (layer, sequence).  q/k/v/ids: the stored inputs (any device);
+    out_*: what the CUDA path produced.  Returns a dict of diagnostics."""
+    kw = params or {}
+    r = oracle.compress(q, k, ids, bitmap, vocab, budget, candidates, **kw)
+    L = k.shape[0]
+    W = q.shape[1]
+    T = L - W
+    n_ref = r["n_keep"]
+    assert int(n_keep) == n_ref, ("n_keep", int(n_keep), n_ref)
+    idx = out_idx[:n_ref].detach().cpu().numpy()
+    info = dict(n_keep=n_ref, margins=r["margins"].copy())
+    if n_ref < L:
+        if s_gpu is not None:
+            info["s_relerr"] = assert_scores_close(s_gpu[:T], r["s"], "s")
+        if e_gpu is not None:
+            info["e_relerr"] = assert_scores_close(e_gpu[:T], r["e"], "e", abs_=1e-4)
+        if sr_gpu is not None:
+            info["sr_relerr"] = assert_scores_close(sr_gpu[:T], r["s_ref"], "s_refined")
+        assert (np.diff(idx) > 0).all(), "indices not strictly ascending"
+        assert idx[-W:].tolist() == list(range(T, L)), "window not retained last"
+        exact = idx.tolist() == r["out_idx"].tolist()
+        info["exact_vs_pure_oracle"] = exact
+        info["overlap"] = len(set(idx.tolist()) & set(r["out_idx"].tolist())) / n_ref
+        if not exact:
+            # tie-aware: allowed only if some decision margin of the pure oracle is below tolerance,
+            # and Algorithm 2 on the GPU's own refined scores reproduces the GPU's indices exactly.
+            assert r["margins"].min() <= 4 * REL, ("indices differ although every margin is wide", r["margins"])
+            assert sr_gpu is not None, "need the GPU's refined scores for the tie-aware check"
+        if sr_gpu is not None:
+            B = n_ref - W
+            sr32 = sr_gpu[:T].detach().cpu().numpy().astype(np.float64)
+            r2 = oracle.select(sr32, r["seg_start"], B, candidates, tau=float(np.float32(kw.get("tau", 0.85))))
+            assert idx[:B].tolist() == r2["keep"].tolist(), "Algorithm 2 on the GPU's scores disagrees with the GPU"
+            # retained refined-score mass within tolerance of the pure oracle's
+            mass_gpu = r["s_ref"][idx[:B]].sum()
+            mass_ref = r["s_ref"][r["out_idx"][:B]].sum()
+            assert abs(mass_gpu - mass_ref) <= 4 * REL * mass_ref + ABS
+    else:
+        assert idx.tolist() == list(range(L))
+    # compaction: byte-exact gather at the (validated) indices
+    for name, src, dst in (("k", k, out_k), ("v", v, out_v)):
+        ref_bytes = oracle.gather(src, idx)
+        got = dst[:n_ref].detach().cpu().contiguous().view(torch.uint8).numpy().reshape(n_ref, -1)
+        assert (got == ref_bytes).all(), f"compacted {name} differs"
+    return info

@@ -1,0 +1,206 @@
+"""Parity of the fused pass (sablock_compress / sablock_compress_layers) against the oracle,
+on the benchmark's configurations and on the method's edge cases (needs a B200)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth
+from paper_2510_22556_b200 import binding as B
+from paper_2510_22556_b200 import build as build_lib
+from parity import check_problem
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build_lib()
+    B.lib()
+
+
+def _params(cfg, bitmap, **kw):
+    return B.make_params(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.window, synth.torch_dtype(cfg.dtype),
+                         bitmap, cfg.vocab, **kw)
+
+
+def run_batch(cfg, batch, budget, layers_to_check=None, **kw):
+    """Runs sablock_compress_layers on a synth.Batch (already on the GPU) and checks the chosen
+    layers of every sequence against the oracle, using the scores the same call left in the
+    workspace for the tie-aware part."""
+    nl, ns = batch.q_win.shape[0], batch.q_win.shape[1]
+    cu = batch.cu_seqlens
+    total, max_L = cu[-1], max(b - a for a, b in zip(cu[:-1], cu[1:]))
+    p = _params(cfg, batch.bitmap, **kw)
+    ws = B.alloc_workspace(p, total, max_L, ns, nl)
+    out = B.compress_layers(p, batch.q_win, batch.k, batch.v, batch.token_ids, cu, budget, cfg.candidates, ws)
+    torch.cuda.synchronize()
+    assert B.read_status(ws) == 0
+    s = B.workspace_view(p, ws, "s", total, max_L, ns, nl)
+    e = B.workspace_view(p, ws, "e", total, max_L, ns, nl)
+    sr = B.workspace_view(p, ws, "s_refined", total, max_L, ns, nl)
+    oparams = {k: float(np.float32(v)) if isinstance(v, float) else v for k, v in kw.items()
+               if k in ("alpha", "eta", "eps", "tau", "pool_kernel", "pool_mode")}
+    infos = []
+    for l in (range(nl) if layers_to_check is None else layers_to_check):
+        for i in range(ns):
+            a, z = cu[i], cu[i + 1]
+            infos.append(check_problem(cfg, batch.q_win[l, i], batch.k[l, a:z], batch.v[l, a:z], batch.token_ids[a:z],
+                                       batch.bitmap, cfg.vocab, budget, cfg.candidates, out.out_k[l, i],
+                                       out.out_v[l, i], out.out_idx[l, i], out.n_keep[l, i].item(),
+                                       s_gpu=s[l, a:z], e_gpu=e[l, a:z], sr_gpu=sr[l, a:z], params=oparams))
+    return out, infos
+
+
+def test_tiny_config():
+    cfg = synth.CONFIGS["tiny"]
+    b = synth.make_batch(cfg, device="cuda")
+    out, infos = run_batch(cfg, b, 64)
+    assert out.n_keep.item() == 64
+
+
+@pytest.mark.parametrize("budget", [96, 128, 256])
+def test_layer8k_config(budget):
+    cfg = synth.CONFIGS["layer8k"]
+    b = synth.make_batch(cfg, device="cuda")
+    out, infos = run_batch(cfg, b, budget)
+    # the planted needle span (keys aligned with the mean window query) survives compression
+    start, n = b.spans[0][0]
+    idx = out.out_idx[0, 0].cpu().numpy()
+    assert ((idx >= start) & (idx < start + n)).sum() >= min(n, budget - cfg.window) // 2
+
+
+def test_single_layer_entry_point_equals_batched():
+    cfg = synth.CONFIGS["layer8k"]
+    b = synth.make_batch(cfg, device="cuda")
+    p = _params(cfg, b.bitmap)
+    ws = B.alloc_workspace(p, 8192, 8192)
+    ok, ov, oi, nk = B.compress(p, b.q_win[0, 0], b.k[0], b.v[0], b.token_ids, 128, cfg.candidates, ws)
+    out = B.compress_layers(p, b.q_win, b.k, b.v, b.token_ids, b.cu_seqlens, 128, cfg.candidates, ws)
+    torch.cuda.synchronize()
+    assert nk.item() == 128
+    assert torch.equal(oi, out.out_idx[0, 0]) and torch.equal(ok, out.out_k[0, 0]) and torch.equal(ov, out.out_v[0, 0])
+
+
+def test_stack32k_layers_and_budget_trend():
+    """Three layers of the 32K stack at two budgets; larger budgets choose larger blocks."""
+    cfg = synth.CONFIGS["stack32k"]
+    b = synth.make_batch(cfg, device="cuda", n_layers=3)
+    for budget in (128, 2048):
+        run_batch(cfg, b, budget, layers_to_check=[0, 2])
+
+
+def test_ragged_batch_small():
+    cfg = synth.CONFIGS["ragged16"]
+    lens = [700, 1300, 515, 4096 + 17, 129]
+    b = synth.make_batch(cfg, device="cuda", n_layers=2, seq_lens=lens)
+    out, infos = run_batch(cfg, b, 128)
+    assert out.n_keep.cpu().tolist() == [[128] * 5] * 2
+
+
+def test_ragged_batch_with_identity_sequences():
+    """Sequences that already fit the budget come back unchanged next to compressed ones."""
+    cfg = synth.CONFIGS["ragged16"]
+    lens = [100, 2000, 512, 513, 31]
+    b = synth.make_batch(cfg, device="cuda", n_layers=2, seq_lens=lens)
+    out, infos = run_batch(cfg, b, 512)
+    assert out.n_keep[0].cpu().tolist() == [100, 512, 512, 512, 31]
+
+
+@pytest.mark.parametrize("impl", [B.SCORE_SIMT, B.SCORE_TENSOR])
+def test_no_delimiters_single_segment(impl):
+    cfg = synth.CONFIGS["layer8k"]
+    b = synth.make_batch(cfg, device="cuda", seq_lens=[3000], with_delimiters=False)
+    run_batch(cfg, b, 256, score_impl=impl)
+
+
+def test_every_token_a_delimiter():
+    cfg = synth.CONFIGS["layer8k"]
+    b = synth.make_batch(cfg, device="cuda", seq_lens=[2000])
+    b.token_ids[:] = synth.delimiter_ids(cfg.vocab)[0]
+    run_batch(cfg, b, 200)
+
+
+@pytest.mark.parametrize("kw", [dict(tau=0.0), dict(tau=1.0), dict(alpha=0.0), dict(eta=0.0, alpha=3.0),
+                                dict(pool_kernel=7, pool_mode=0), dict(budget_includes_window=0)])
+def test_parameter_variants(kw):
+    cfg = synth.CONFIGS["layer8k"]
+    b = synth.make_batch(cfg, device="cuda", seq_lens=[4096])
+    if "budget_includes_window" in kw:
+        p = _params(cfg, b.bitmap, **kw)
+        ws = B.alloc_workspace(p, 4096, 4096)
+        out = B.compress_layers(p, b.q_win, b.k, b.v, b.token_ids, b.cu_seqlens, 100, cfg.candidates, ws)
+        torch.cuda.synchronize()
+        assert out.n_keep.item() == 100 + cfg.window
+        r = oracle.compress(b.q_win[0, 0], b.k[0], b.token_ids, b.bitmap, cfg.vocab, 100 + cfg.window, cfg.candidates)
+        assert len(set(out.out_idx[0, 0].cpu().tolist()) & set(r["out_idx"].tolist())) >= 0.95 * (100 + cfg.window)
+        return
+    run_batch(cfg, b, 160, **kw)
+
+
+def test_paper_defaults_window8_candidates():
+    """The paper's own settings: n_rcnt = 8, search set {1,2,3,5,7,9,11,13} (Sec. 4.1, Sec. 4.5)."""
+    cfg = synth.Config("paper", 1, 32, 8, 128, 8, (6000,), (96,), (1, 2, 3, 5, 7, 9, 11, 13), "bf16", 128256, 16, 2.0,
+                       25, (0.3,), 11)
+    b = synth.make_batch(cfg, device="cuda")
+    run_batch(cfg, b, 96)
+    run_batch(cfg, b, 1024)
+
+
+def test_strided_kv_cache():
+    """K/V stored as one interleaved [L, 2, Hkv, D] buffer (token stride twice the row)."""
+    cfg = synth.CONFIGS["layer8k"]
+    b = synth.make_batch(cfg, device="cuda", seq_lens=[2500])
+    kv = torch.stack([b.k[0], b.v[0]], dim=1).contiguous()            # [L, 2, Hkv, D]
+    tok = 2 * cfg.n_kv_heads * cfg.head_dim
+    p = _params(cfg, b.bitmap, k_stride_token=tok, v_stride_token=tok)
+    ws = B.alloc_workspace(p, 2500, 2500)
+    ok, ov, oi, nk = B.compress(p, b.q_win[0, 0], kv[:, 0], kv[:, 1], b.token_ids, 128, cfg.candidates, ws)
+    p2 = _params(cfg, b.bitmap)
+    ok2, ov2, oi2, nk2 = B.compress(p2, b.q_win[0, 0], b.k[0], b.v[0], b.token_ids, 128, cfg.candidates, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(oi, oi2) and torch.equal(ok, ok2) and torch.equal(ov, ov2)
+
+
+def test_host_buffer_entry_point():
+    cfg = synth.CONFIGS["layer8k"]
+    b = synth.make_batch(cfg, device="cpu", seq_lens=[2048, 1000], n_layers=2)
+    d = synth.make_batch(cfg, device="cpu", seq_lens=[2048, 1000], n_layers=2)
+    p = _params(cfg, b.bitmap.cuda())
+    total, max_L = b.cu_seqlens[-1], 2048
+    ws = B.alloc_workspace(p, total, max_L, 2, 2)
+    pin = lambda t: t.pin_memory()
+    hq, hk, hv, hid = pin(b.q_win), pin(b.k), pin(b.v), pin(b.token_ids)
+    dq, dk, dv, did = (torch.empty_like(t, device="cuda") for t in (hq, hk, hv, hid))
+    h_out = B.LayersOut(p, 2, 2, 128, hk.dtype, pinned_host=True)
+    d_out = B.LayersOut(p, 2, 2, 128, hk.dtype)
+    B.compress_layers_host(p, hq, hk, hv, hid, b.cu_seqlens, 128, cfg.candidates, h_out, dq, dk, dv, did, d_out, ws)
+    ref = B.compress_layers(p, d.q_win.cuda(), d.k.cuda(), d.v.cuda(), d.token_ids.cuda(), d.cu_seqlens, 128,
+                            cfg.candidates, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(h_out.out_idx, ref.out_idx.cpu()) and torch.equal(h_out.out_k, ref.out_k.cpu())
+    assert torch.equal(h_out.out_v, ref.out_v.cpu()) and h_out.n_keep.tolist() == [[128, 128]] * 2
+
+
+def test_headline_config_full_size():
+    """The benchmark's launch configuration: 32 layers x 131072 tokens, budget 1024.  Layers 0 and
+    31 are checked against the oracle in full; every layer is checked for the invariants."""
+    cfg = synth.CONFIGS["headline128k"]
+    b = synth.make_batch(cfg, device="cuda")
+    out, infos = run_batch(cfg, b, 1024, layers_to_check=[0, 31])
+    idx = out.out_idx[:, 0].cpu().numpy()
+    L, W = cfg.seq_lens[0], cfg.window
+    assert (out.n_keep.cpu().numpy() == 1024).all()
+    assert (np.diff(idx, axis=1) > 0).all()
+    assert (idx[:, -W:] == np.arange(L - W, L)[None]).all()
+    # compacted rows of every layer are the input rows at the chosen positions
+    for l in range(cfg.n_layers):
+        sel = torch.from_numpy(idx[l]).cuda().long()
+        assert torch.equal(out.out_k[l, 0], b.k[l, sel]) and torch.equal(out.out_v[l, 0], b.v[l, sel])
+
+
+def test_ragged16_config_full_size():
+    cfg = synth.CONFIGS["ragged16"]
+    b = synth.make_batch(cfg, device="cuda")
+    out, infos = run_batch(cfg, b, 512, layers_to_check=[7])
+    assert (out.n_keep.cpu().numpy() == 512).all()
