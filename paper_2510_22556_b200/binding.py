@@ -67,6 +67,8 @@ def lib():
         l.sablock_workspace_bytes.argtypes = [C.c_void_p, C.c_longlong, C.c_int, C.c_int, C.c_int]
         vp, ci, sz = C.c_void_p, C.c_int, C.c_size_t
         l.sablock_read_status.argtypes = [vp, vp, vp]
+        l.sablock_workspace_region.argtypes = [vp, C.c_longlong, ci, ci, ci, C.c_char_p, vp, vp]
+        l.sablock_params_default.argtypes = [vp]
         l.sablock_segment.argtypes = [vp, vp, ci, vp, vp, vp, vp, sz, vp]
         l.sablock_score.argtypes = [vp, vp, vp, ci, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         l.sablock_select.argtypes = [vp, vp, ci, vp, vp, ci, vp, ci, vp, vp, vp, vp, sz, vp]
@@ -99,7 +101,7 @@ def _iarr(xs: Sequence[int]):
 def make_params(n_q_heads: int, n_kv_heads: int, head_dim: int, window: int, dtype: torch.dtype,
                 delim_bitmap: Optional[torch.Tensor] = None, vocab_size: int = 0, **kw) -> Params:
     p = Params()
-    lib().sablock_params_default(C.byref(p))
+    lib().sablock_params_default(C.addressof(p))
     p.n_q_heads, p.n_kv_heads, p.head_dim, p.window = n_q_heads, n_kv_heads, head_dim, window
     p.dtype = {torch.float32: F32, torch.bfloat16: BF16}[dtype]
     if delim_bitmap is not None:
@@ -124,8 +126,8 @@ def workspace_view(p: Params, ws: torch.Tensor, name: str, total_tokens: int, ma
                    n_layers: int = 1) -> torch.Tensor:
     """A typed view of one of the fused call's intermediate arrays inside the workspace."""
     off, nb = C.c_size_t(0), C.c_size_t(0)
-    _check(lib().sablock_workspace_region(C.addressof(p), C.c_longlong(total_tokens), max_L, n_seqs, n_layers,
-                                          name.encode(), C.byref(off), C.byref(nb)), "sablock_workspace_region")
+    _check(lib().sablock_workspace_region(C.addressof(p), total_tokens, max_L, n_seqs, n_layers, name.encode(),
+                                          C.addressof(off), C.addressof(nb)), "sablock_workspace_region")
     raw = ws[off.value: off.value + nb.value]
     dt = torch.float32 if name in ("s", "e", "s_refined") else torch.int32
     v = raw.view(dt)

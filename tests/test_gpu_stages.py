@@ -28,12 +28,12 @@ def _sync_ok(ws):
 # ------------------------------------------------------------------ stage 1
 @pytest.mark.parametrize("L,W,gap,delims", [
     (512, 16, 20, True), (8192, 32, 25, True), (5000, 32, 3, True), (70001, 8, 25, True),
-    (4096, 32, 25, False), (2049 + 32, 32, 1, True), (33, 32, 2, True), (131072, 32, 25, True),
+    (4096, 32, 25, False), (2049 + 32, 32, -1, True), (33, 32, 2, True), (131072, 32, 25, True),
 ])
 def test_segment_bit_exact(L, W, gap, delims):
     vocab = 128256
-    ids = synth.make_token_ids(L, vocab, gap, seed=L + W, with_delimiters=delims)
-    if gap == 1:                                        # every token a delimiter
+    ids = synth.make_token_ids(L, vocab, abs(gap) + 1, seed=L + W, with_delimiters=delims)
+    if gap < 0:                                         # every token a delimiter
         ids[:] = synth.delimiter_ids(vocab)[0]
     bm = synth.delimiter_bitmap(vocab)
     ref_id, ref_start = oracle.segment(ids, W, bm, vocab)

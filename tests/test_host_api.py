@@ -32,7 +32,7 @@ def test_exports_every_declared_symbol(lib):
 
 def test_defaults_follow_the_paper(lib):
     p = B.Params()
-    lib.sablock_params_default(C.byref(p))
+    lib.sablock_params_default(C.addressof(p))
     assert (round(p.alpha, 6), round(p.eta, 6), round(p.tau, 6)) == (0.9, 1.0, 0.85)
     assert abs(p.eps - 1e-6) < 1e-12
     assert p.pool_kernel == 1 and p.budget_includes_window == 1
@@ -104,3 +104,23 @@ def test_binding_fails_loudly_without_library(monkeypatch):
     monkeypatch.setattr(B, "LIB_PATH", "/nonexistent/libsablock.so")
     with pytest.raises(ImportError):
         B.lib()
+
+
+def test_workspace_regions(lib):
+    p = _params()
+    total = B.workspace_bytes(p, 20000, 8192, 3, 2)
+    seen = []
+    for name in ("s", "e", "s_refined", "seg_id", "seg_start", "n_seg"):
+        off, nb = C.c_size_t(0), C.c_size_t(0)
+        st = lib.sablock_workspace_region(C.addressof(p), 20000, 8192, 3, 2, name.encode(), C.addressof(off),
+                                          C.addressof(nb))
+        assert st == 0 and off.value % 256 == 0 and off.value + nb.value <= total
+        seen.append((off.value, off.value + nb.value))
+    seen.sort()
+    assert all(a[1] <= b[0] for a, b in zip(seen, seen[1:]))          # regions do not overlap
+    off, nb = C.c_size_t(0), C.c_size_t(0)
+    assert lib.sablock_workspace_region(C.addressof(p), 20000, 8192, 3, 2, b"nope", C.addressof(off),
+                                        C.addressof(nb)) == 1
+    ws = torch.zeros(total, dtype=torch.uint8)
+    v = B.workspace_view(p, ws, "s_refined", 20000, 8192, 3, 2)
+    assert v.shape == (2, 20000) and v.dtype == torch.float32
