@@ -1,0 +1,355 @@
+#!/usr/bin/env python
+"""Benchmark of the SABlock prefill-time KV-cache compression pass on B200.
+
+One "step" is one pass of the whole hot path (segmentation, window scoring, refinement,
+block-size search, top-k, compaction) over the headline workload: 32 layers of a
+Llama-3-8B-shaped KV cache at 131072 tokens, budget 1024 (synthetic, seeded).  The metric
+is context tokens compressed per second (tokens of context / time of the 32-layer pass).
+
+  python bench.py --gpus 1 --steps K --warmup W          # CUDA library (this repo)
+  python bench.py --impl reference --steps K --warmup W   # the float64 CPU oracle, timed
+
+With N > 1 (launched by torch.distributed.run) every rank compresses its own replica of the
+workload: the pass has no exchange step, so there is no data-path collective.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch
+
+import synth
+
+METRIC = "context tokens compressed/sec at 128K, budget 1024 (32 layers)"
+UNIT = "tokens/s"
+WORKLOAD = "headline128k"
+BUDGET = 1024
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), float(d.get("bf16_tflops_sustained", d.get("bf16_tflops", 1378.0))), "measured"
+    return 6650.0, 1400.0, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, device_index: int, period_s: float = 0.02):
+        super().__init__(daemon=True)
+        self.period = period_s
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            handle = None
+            try:
+                uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+                for cand in (uuid, "GPU-" + uuid):
+                    try:
+                        handle = pynvml.nvmlDeviceGetHandleByUUID(cand.encode() if isinstance(cand, str) else cand)
+                        break
+                    except Exception:
+                        handle = None
+            except Exception:
+                handle = None
+            if handle is None:
+                visible = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+                idx = device_index
+                if visible and all(v.strip().isdigit() for v in visible.split(",")):
+                    idx = int(visible.split(",")[device_index])
+                handle = pynvml.nvmlDeviceGetHandleByIndex(idx)
+            self.h = handle
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(handle, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+            getattr(nv, "nvmlClocksEventReasonHwPowerBrakeSlowdown", 0x80): "hw_power_brake",
+        }
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                try:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=2)
+        s = sorted(self.samples)
+        return {"sm_mhz": (s[len(s) // 2] if s else None), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(s)}
+
+
+def algorithmic_bytes(cfg, n_layers, L, n_out):
+    """Bytes the method must move for one sequence (K read once, q_win, token ids, gather r/w)."""
+    es = 2 if cfg.dtype == "bf16" else 4
+    row = cfg.n_kv_heads * cfg.head_dim * es
+    k_read = n_layers * L * row
+    gather = n_layers * 4 * n_out * row
+    q = n_layers * cfg.n_q_heads * cfg.window * cfg.head_dim * es
+    return dict(k_read=k_read, total=k_read + gather + q + n_layers * n_out * 4 + L * 4)
+
+
+def run_ours(args):
+    from paper_2510_22556_b200 import binding as B
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl")
+    B.lib()          # fails loudly if the CUDA library is missing: there is no fallback
+    cfg = synth.CONFIGS[args.workload]
+    nl = cfg.n_layers if args.layers is None else args.layers
+    batch = synth.make_batch(cfg, device="cuda", n_layers=nl)
+    cu = batch.cu_seqlens
+    total, max_L, ns = cu[-1], max(b - a for a, b in zip(cu[:-1], cu[1:])), len(cu) - 1
+    budget = args.budget
+    p = B.make_params(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.window, batch.k.dtype, batch.bitmap, cfg.vocab)
+    ws = B.alloc_workspace(p, total, max_L, ns, nl)
+    out = B.LayersOut(p, nl, ns, budget, batch.k.dtype)
+
+    def step():
+        B.compress_layers(p, batch.q_win, batch.k, batch.v, batch.token_ids, cu, budget, cfg.candidates, ws, out)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    assert B.read_status(ws) == 0, "device status word set during warm-up"
+
+    slots = min(args.steps, 512)
+    B.profile_enable(slots)
+    sampler = ClockSampler(local)
+    sampler.start()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches = 0
+    ev0.record()
+    for _ in range(args.steps):
+        step()
+        launches += B.last_launch_count()
+    ev1.record()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    clocks = sampler.stop()
+    ms_total = ev0.elapsed_time(ev1)
+    if dist is not None:
+        t = torch.tensor([ms_total], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    assert B.read_status(ws) == 0, "device status word set during the timed region"
+    stage_ms = {}
+    for s in range(slots):
+        for name, ms in B.profile_read(s).items():
+            stage_ms.setdefault(name, []).append(ms)
+    B.profile_enable(0)
+    stage_avg = {k: sum(v) / len(v) for k, v in stage_ms.items()}
+
+    tokens = total                               # context tokens per step on this rank
+    value = world * tokens / (ms_step * 1e-3)
+
+    # ---- roofline of the dominant kernel (one launch per step each) ------------------------
+    hbm_peak, tf_peak, peak_src = measured_peaks()
+    ab = algorithmic_bytes(cfg, nl, total, out.n_out)
+    dom = max(("score_pass1", "score_pass2"), key=lambda k: stage_avg.get(k, 0.0))
+    dom_ms = stage_avg.get(dom, float("nan"))
+    achieved = ab["k_read"] / (dom_ms * 1e-3) / 1e9
+    traffic = TRAFFIC_BYTES_PER_LAUNCH.get(dom)
+    if traffic is not None:
+        traffic = traffic * (nl * total) / TRAFFIC_CAPTURE_TOKEN_LAYERS
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": round(achieved, 1), "peak": hbm_peak, "unit": "GB/s",
+                "frac": round(achieved / hbm_peak, 4), "traffic": traffic, "peak_source": peak_src,
+                "launch_ms": round(dom_ms, 4)}
+    flops = 2.0 * cfg.n_q_heads * cfg.window * cfg.head_dim * total * nl
+    t_roof_ms = max(ab["total"] / (hbm_peak * 1e9), flops / (tf_peak * 1e12)) * 1e3
+    path = {"t_roofline_ms": round(t_roof_ms, 4), "frac_of_measured_hbm": round(t_roof_ms / ms_step, 4),
+            "frac_of_nominal_8TBs": round(ab["total"] / 8e12 * 1e3 / ms_step, 4),
+            "algorithmic_bytes": ab["total"], "score_flops": flops,
+            "stage_ms": {k: round(v, 4) for k, v in stage_avg.items()}}
+
+    result = {
+        "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": round(ms_step, 4), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "n_layers": nl, "seq_len": max_L, "n_seqs": ns, "budget": budget,
+                   "window": cfg.window, "n_q_heads": cfg.n_q_heads, "n_kv_heads": cfg.n_kv_heads,
+                   "head_dim": cfg.head_dim, "candidates": list(cfg.candidates),
+                   "l2": "inputs larger than L2 (K alone is %.1f GB per step)" % (ab["k_read"] / 1e9),
+                   "multi_gpu": "replicas only"},
+        "clocks": clocks, "gpu_launches": launches, "roofline": roofline, "roofline_path": path,
+    }
+
+    if rank == 0 and world == 1 and not args.no_e2e:
+        result["e2e"] = run_e2e(B, cfg, batch, p, ws, out, budget, args)
+    elif rank == 0:
+        result["e2e"] = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        result["cpu_baseline"] = cpu_baseline(cfg, batch, budget, nl, target_s=15.0)
+    if rank == 0:
+        print(json.dumps(result))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+# DRAM bytes (read + write) per launch from the ncu capture summarised under profiles/,
+# taken on a smaller case and scaled by (layers x tokens); None until captured.
+TRAFFIC_BYTES_PER_LAUNCH = {}
+TRAFFIC_CAPTURE_TOKEN_LAYERS = 1
+
+
+def run_e2e(B, cfg, batch, p, ws, out, budget, args):
+    """Same metric through the host-buffer entry point: pinned host inputs are copied to the
+    device, compressed, and the compacted cache is copied back, all inside the timed region."""
+    nl, ns = batch.q_win.shape[0], batch.q_win.shape[1]
+    cu = batch.cu_seqlens
+    hq, hk, hv, hid = (t.cpu().pin_memory() for t in (batch.q_win, batch.k, batch.v, batch.token_ids))
+    h_out = B.LayersOut(p, nl, ns, budget, batch.k.dtype, pinned_host=True)
+    steps = max(1, min(args.e2e_steps, args.steps))
+
+    def step():
+        B.compress_layers_host(p, hq, hk, hv, hid, cu, budget, cfg.candidates, h_out, batch.q_win, batch.k, batch.v,
+                               batch.token_ids, out, ws)
+
+    step()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        step()                      # returns after the stream has drained (results are on the host)
+    dt = (time.perf_counter() - t0) / steps
+    h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv, hid))
+    d2h = sum(t.numel() * t.element_size() for t in (h_out.out_k, h_out.out_v, h_out.out_idx, h_out.n_keep))
+    assert int(h_out.n_keep.min()) == out.n_out
+    return {"value": round(cu[-1] / dt, 1), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "ms_per_step": round(dt * 1e3, 3), "steps": steps}
+
+
+def oracle_sample(cfg, q, k, ids, bitmap, budget, L_sample):
+    """Times the oracle, as it stands, on the first L_sample tokens of one layer."""
+    import oracle
+    W = cfg.window
+    qs = q.cpu()
+    ks = k[:L_sample].cpu()
+    # the window queries stay the layer's own; the sample is a shorter prompt of the same kind
+    t0 = time.perf_counter()
+    oracle.compress(qs, ks, ids[:L_sample].cpu(), bitmap.cpu(), cfg.vocab, min(budget, L_sample - 1), cfg.candidates)
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(cfg, batch, budget, n_layers, target_s=15.0):
+    import oracle
+    cu = batch.cu_seqlens
+    L = cu[1] - cu[0]
+    q, k, ids = batch.q_win[0, 0], batch.k[0, :L], batch.token_ids[:L]
+    t_small = oracle_sample(cfg, q, k, ids, batch.bitmap, budget, 4096)       # also warms the library
+    t_small = oracle_sample(cfg, q, k, ids, batch.bitmap, budget, 4096)
+    L_s = int(min(L, max(4096, 4096 * target_s / max(t_small, 1e-4))))
+    L_s = (L_s // 1024) * 1024
+    t = oracle_sample(cfg, q, k, ids, batch.bitmap, budget, L_s)
+    cores = min(oracle.num_threads(), cfg.window)
+    value = L_s / (t * n_layers)          # one layer timed; the metric's pass has n_layers of them
+    return {"value": round(value, 2), "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"float64 oracle on the first {L_s} tokens of layer 0 ({t:.2f} s), x{n_layers} layers extrapolated"}
+
+
+def run_reference(args):
+    """The reference arm: the oracle timed on the host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import oracle
+    cfg = synth.CONFIGS[args.workload]
+    nl = cfg.n_layers if args.layers is None else args.layers
+    L = cfg.seq_lens[0]
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    q, k, v, _ = synth.make_layer(cfg, L, synth.layer_seed(cfg, 0, 0), device=dev)
+    ids = synth.make_token_ids(L, cfg.vocab, cfg.mean_gap, synth.token_seed(cfg, 0))
+    bitmap = synth.delimiter_bitmap(cfg.vocab)
+    q, k = q.cpu(), k.cpu()
+    t_small = oracle_sample(cfg, q, k, ids, bitmap, args.budget, 4096)
+    t_small = oracle_sample(cfg, q, k, ids, bitmap, args.budget, 4096)
+    n_calls = args.steps + args.warmup
+    per_step = max(0.2, 150.0 / n_calls)                      # whole run within a few minutes
+    L_s = int(min(L, max(2048, 4096 * per_step / max(t_small, 1e-4))))
+    L_s = max(2048, (L_s // 1024) * 1024)
+    for _ in range(args.warmup):
+        oracle_sample(cfg, q, k, ids, bitmap, args.budget, L_s)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_sample(cfg, q, k, ids, bitmap, args.budget, L_s)
+    dt = (time.perf_counter() - t0) / args.steps
+    value = L_s / (dt * nl)
+    cores = min(oracle.num_threads(), cfg.window)
+    sample = f"float64 oracle on the first {L_s} tokens of one layer per step, x{nl} layers extrapolated"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": round(value, 2), "unit": UNIT,
+        "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": round(dt * 1e3, 3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "n_layers": nl, "seq_len": L, "budget": args.budget, "sample": sample},
+        "cpu_baseline": {"value": round(value, 2), "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": round(value, 2), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=WORKLOAD, choices=list(synth.CONFIGS))
+    ap.add_argument("--budget", type=int, default=BUDGET)
+    ap.add_argument("--layers", type=int, default=None, help="override the number of layers (profiling small cases)")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

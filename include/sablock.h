@@ -185,6 +185,18 @@ sablock_status_t sablock_compress_layers_host(const sablock_params_t *p, int n_l
                                               int *dev_out_n_keep,
                                               void *ws, size_t ws_bytes, sablock_stream_t stream);
 
+/* Per-stage timing (optional, for benchmarks).  While enabled, every fused call of this
+ * thread records CUDA events on its stream between the stages, into the next of `slots`
+ * event sets (round robin; the events are created on first use and kept until exit).
+ * sablock_profile_read(slot, ...) waits for that slot's last event and stores the
+ * milliseconds of each stage interval; it returns the number of intervals (0 if the slot
+ * was never used).  sablock_profile_stage_name(i) names interval i.  The stages are:
+ * segment, score_pass1, score_merge, score_pass2, refine, topb, search, index, compact. */
+#define SABLOCK_PROFILE_MAX_SLOTS 512
+sablock_status_t sablock_profile_enable(int slots);   /* 0 disables; resets the slot counter */
+int sablock_profile_read(int slot, float *ms_out, int max_n);
+const char *sablock_profile_stage_name(int i);
+
 /* Number of kernels the most recent entry-point call of this thread enqueued (for
  * launch accounting in benchmarks). */
 int sablock_last_launch_count(void);

@@ -25,7 +25,8 @@ EXPORTS = [
     "sablock_params_default", "sablock_status_string", "sablock_version", "sablock_workspace_bytes",
     "sablock_read_status", "sablock_segment", "sablock_score", "sablock_select", "sablock_compact",
     "sablock_compress", "sablock_compress_layers", "sablock_compress_layers_host", "sablock_last_launch_count",
-    "sablock_params_sizeof", "sablock_workspace_region",
+    "sablock_params_sizeof", "sablock_workspace_region", "sablock_profile_enable", "sablock_profile_read",
+    "sablock_profile_stage_name",
 ]
 
 
@@ -69,6 +70,8 @@ def lib():
         l.sablock_read_status.argtypes = [vp, vp, vp]
         l.sablock_workspace_region.argtypes = [vp, C.c_longlong, ci, ci, ci, C.c_char_p, vp, vp]
         l.sablock_params_default.argtypes = [vp]
+        l.sablock_profile_read.argtypes = [ci, vp, ci]
+        l.sablock_profile_stage_name.restype = C.c_char_p
         l.sablock_segment.argtypes = [vp, vp, ci, vp, vp, vp, vp, sz, vp]
         l.sablock_score.argtypes = [vp, vp, vp, ci, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         l.sablock_select.argtypes = [vp, vp, ci, vp, vp, ci, vp, ci, vp, vp, vp, vp, sz, vp]
@@ -143,6 +146,17 @@ def read_status(ws: torch.Tensor) -> int:
     raw = C.c_int(0)
     code = lib().sablock_read_status(_ptr(ws), _stream(), C.addressof(raw))
     return code
+
+
+def profile_enable(slots: int) -> None:
+    _check(lib().sablock_profile_enable(int(slots)), "sablock_profile_enable")
+
+
+def profile_read(slot: int):
+    """Stage name -> milliseconds for the fused call that used event slot `slot`."""
+    buf = (C.c_float * 16)()
+    n = lib().sablock_profile_read(slot, C.addressof(buf), 16)
+    return {lib().sablock_profile_stage_name(i).decode(): float(buf[i]) for i in range(n)}
 
 
 def last_launch_count() -> int:

@@ -16,6 +16,38 @@ namespace {
 
 thread_local int t_launches = 0;
 
+// ---- optional per-stage event timing ---------------------------------------------------
+constexpr int kProfStages = 9;
+const char* const kProfNames[kProfStages] = {"segment", "score_pass1", "score_merge", "score_pass2", "refine",
+                                             "topb", "search", "index", "compact"};
+struct ProfState {
+    int slots = 0, next = 0, cur = -1;
+    cudaEvent_t ev[SABLOCK_PROFILE_MAX_SLOTS][kProfStages + 1] = {};
+    bool used[SABLOCK_PROFILE_MAX_SLOTS] = {};
+};
+thread_local ProfState* t_prof = nullptr;
+
+void prof_begin_call(cudaStream_t st)
+{
+    if (!t_prof || t_prof->slots <= 0) return;
+    ProfState& ps = *t_prof;
+    ps.cur = ps.next;
+    ps.next = (ps.next + 1) % ps.slots;
+    for (int i = 0; i <= kProfStages; ++i)
+        if (!ps.ev[ps.cur][i]) cudaEventCreate(&ps.ev[ps.cur][i]);
+    ps.used[ps.cur] = true;
+    cudaEventRecord(ps.ev[ps.cur][0], st);
+}
+void prof_mark(int stage_done, cudaStream_t st)      // after stage `stage_done` (0-based)
+{
+    if (!t_prof || t_prof->slots <= 0 || t_prof->cur < 0) return;
+    cudaEventRecord(t_prof->ev[t_prof->cur][stage_done + 1], st);
+}
+void prof_end_call()
+{
+    if (t_prof) t_prof->cur = -1;
+}
+
 inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 
 struct Plan {
@@ -269,8 +301,10 @@ sablock_status_t run_score(const Plan& pl, const sablock_params_t* p, const void
         dim3 grid1(pl.n_chunks, g.Hkv, pl.n_prob);
         k1<<<grid1, kTcThreads, smem1, stream>>>(tmQ, tmK, g, c2, sb, pl.tpc1, status);
         SAB_TRY(check_launch());
+        prof_mark(1, stream);
         lse_merge_tc<<<dim3(g.Hkv, pl.n_prob), 128, 0, stream>>>(g, sb, pl.tpc1);
         SAB_TRY(check_launch());
+        prof_mark(2, stream);
         switch (g.window) {
             case 8: return launch_p2_tc<8>(pl, tmQ, tmK, c2, p->eps, sb, s, e, status, stream);
             case 16: return launch_p2_tc<16>(pl, tmQ, tmK, c2, p->eps, sb, s, e, status, stream);
@@ -290,8 +324,10 @@ sablock_status_t run_score(const Plan& pl, const sablock_params_t* p, const void
         k1<<<grid1, kSimtThreads, smem1, stream>>>(g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, ks.tok, ks.head,
                                                    ks.layer, c2, sb);
         SAB_TRY(check_launch());
+        prof_mark(1, stream);
         lse_merge_simt<<<gridm, 128, 0, stream>>>(g, sb);
         SAB_TRY(check_launch());
+        prof_mark(2, stream);
         score_p2_simt<__nv_bfloat16><<<grid2, kSimtThreads, smem2, stream>>>(
             g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, ks.tok, ks.head, ks.layer, c2, p->eps, sb, s, e);
     } else {
@@ -300,8 +336,10 @@ sablock_status_t run_score(const Plan& pl, const sablock_params_t* p, const void
             return SABLOCK_ERR_CUDA;
         k1<<<grid1, kSimtThreads, smem1, stream>>>(g, (const float*)q, (const float*)k, ks.tok, ks.head, ks.layer, c2, sb);
         SAB_TRY(check_launch());
+        prof_mark(1, stream);
         lse_merge_simt<<<gridm, 128, 0, stream>>>(g, sb);
         SAB_TRY(check_launch());
+        prof_mark(2, stream);
         score_p2_simt<float><<<grid2, kSimtThreads, smem2, stream>>>(g, (const float*)q, (const float*)k, ks.tok,
                                                                      ks.head, ks.layer, c2, p->eps, sb, s, e);
     }
@@ -343,6 +381,7 @@ sablock_status_t run_select(const Plan& pl, const sablock_params_t* p, const flo
     int* cut = at<int>(ws, pl.o_cut);
     topb_kernel<<<pl.n_prob, kTopThreads, 0, stream>>>(g, s_ref, thr, cut);
     SAB_TRY(check_launch());
+    prof_mark(5, stream);
     SearchOut so;
     so.keep = at<unsigned>(ws, pl.o_keep);
     so.keep_words = pl.keep_words;
@@ -357,6 +396,7 @@ sablock_status_t run_select(const Plan& pl, const sablock_params_t* p, const flo
     search_long_kernel<<<dim3(4, pl.n_prob), kLongThreads, 0, stream>>>(g, cands, s_ref, seg_start, thr, cut, p->tau, so,
                                                                        at<double>(ws, pl.o_phi), at<int>(ws, pl.o_rank));
     SAB_TRY(check_launch());
+    prof_mark(6, stream);
     index_kernel<<<pl.n_prob, kIdxThreads, 0, stream>>>(g, so.keep, pl.keep_words, out_idx, out_n_keep,
                                                         at<int>(ws, pl.o_status));
     return check_launch();
@@ -425,6 +465,33 @@ int sablock_version(void) { return 100; }
 size_t sablock_params_sizeof(void) { return sizeof(sablock_params_t); }
 
 int sablock_last_launch_count(void) { return t_launches; }
+
+sablock_status_t sablock_profile_enable(int slots)
+{
+    if (slots < 0 || slots > SABLOCK_PROFILE_MAX_SLOTS) return SABLOCK_ERR_INVALID_ARG;
+    if (!t_prof) {
+        if (slots == 0) return SABLOCK_OK;
+        t_prof = new ProfState();
+    }
+    t_prof->slots = slots;
+    t_prof->next = 0;
+    t_prof->cur = -1;
+    for (int i = 0; i < SABLOCK_PROFILE_MAX_SLOTS; ++i) t_prof->used[i] = false;
+    return SABLOCK_OK;
+}
+
+int sablock_profile_read(int slot, float* ms_out, int max_n)
+{
+    if (!t_prof || slot < 0 || slot >= SABLOCK_PROFILE_MAX_SLOTS || !t_prof->used[slot] || !ms_out) return 0;
+    ProfState& ps = *t_prof;
+    if (cudaEventSynchronize(ps.ev[slot][kProfStages]) != cudaSuccess) return 0;
+    int n = max_n < kProfStages ? max_n : kProfStages;
+    for (int i = 0; i < n; ++i)
+        if (cudaEventElapsedTime(&ms_out[i], ps.ev[slot][i], ps.ev[slot][i + 1]) != cudaSuccess) ms_out[i] = -1.f;
+    return n;
+}
+
+const char* sablock_profile_stage_name(int i) { return (i >= 0 && i < kProfStages) ? kProfNames[i] : ""; }
 
 size_t sablock_workspace_bytes(const sablock_params_t* p, long long total_tokens, int max_L, int n_seqs, int n_layers)
 {
@@ -560,6 +627,7 @@ sablock_status_t sablock_compress_layers(const sablock_params_t* p, int n_layers
     SAB_TRY(make_plan(p, n_layers, n_seqs, cu_seqlens, cu_seqlens[n_seqs], max_L, rows_out(p, budget), &pl));
     if (!ws || ws_bytes < pl.total) return SABLOCK_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    prof_begin_call(st);
     SAB_TRY(zero_control(pl, ws, st));
     int* seg_id = at<int>(ws, pl.o_seg_id);
     int* seg_start = at<int>(ws, pl.o_seg_start);
@@ -569,10 +637,17 @@ sablock_status_t sablock_compress_layers(const sablock_params_t* p, int n_layers
     float* sr = at<float>(ws, pl.o_sr);
     float* s_raw = p->pool_kernel > 1 ? at<float>(ws, pl.o_s_raw) : s;
     SAB_TRY(run_segment(pl, p, token_ids, seg_id, seg_start, n_seg, ws, st));
+    prof_mark(0, st);
     SAB_TRY(run_score(pl, p, q_win, k, s_raw, e, ws, st));
+    prof_mark(3, st);
     SAB_TRY(run_refine(pl, p, s_raw, s, e, seg_start, n_seg, sr, nullptr, 0, st));
+    prof_mark(4, st);
     SAB_TRY(run_select(pl, p, sr, seg_start, n_seg, cands, out_idx, out_n_keep, nullptr, nullptr, 0, ws, st));
-    return run_compact(pl.geo, pl.n_prob, p, k, v, out_idx, out_n_keep, 0, out_k, out_v, st);
+    prof_mark(7, st);
+    sablock_status_t rc = run_compact(pl.geo, pl.n_prob, p, k, v, out_idx, out_n_keep, 0, out_k, out_v, st);
+    prof_mark(8, st);
+    prof_end_call();
+    return rc;
 }
 
 sablock_status_t sablock_compress(const sablock_params_t* p, const void* q_win, const void* k, const void* v,
