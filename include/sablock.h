@@ -43,9 +43,13 @@ typedef enum {
 
 typedef enum { SABLOCK_F32 = 0, SABLOCK_BF16 = 1 } sablock_dtype_t;
 
-/* Which kernel family computes the attention scores. AUTO picks the tensor-core
- * (tcgen05) kernels whenever the shape allows it and the SIMT kernels otherwise. */
-typedef enum { SABLOCK_SCORE_AUTO = 0, SABLOCK_SCORE_SIMT = 1, SABLOCK_SCORE_TENSOR = 2 } sablock_score_impl_t;
+/* Which kernel family computes the attention scores.  AUTO picks, in this order, the
+ * persistent two-sweep tensor-core kernel (bf16, head_dim 128, window 32, four query heads
+ * per KV head, at most 7 token tiles of 128 per CTA), the two-launch tensor-core kernels
+ * (bf16, head_dim 64/128, window 8/16/32), and the SIMT kernels otherwise.  FUSED and TENSOR
+ * force the first and the second and fail with SABLOCK_ERR_UNSUPPORTED where they cannot run. */
+typedef enum { SABLOCK_SCORE_AUTO = 0, SABLOCK_SCORE_SIMT = 1, SABLOCK_SCORE_TENSOR = 2, SABLOCK_SCORE_FUSED = 3 }
+    sablock_score_impl_t;
 
 #define SABLOCK_MAX_SEQS 64        /* sequences per batched call              */
 #define SABLOCK_MAX_CANDIDATES 16  /* block-size candidates                   */

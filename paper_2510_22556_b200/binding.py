@@ -19,7 +19,7 @@ OK = 0
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "WORKSPACE_TOO_SMALL", 4: "CUDA", 5: "TIMEOUT",
                 6: "INTERNAL"}
 F32, BF16 = 0, 1
-SCORE_AUTO, SCORE_SIMT, SCORE_TENSOR = 0, 1, 2
+SCORE_AUTO, SCORE_SIMT, SCORE_TENSOR, SCORE_FUSED = 0, 1, 2, 3
 
 EXPORTS = [
     "sablock_params_default", "sablock_status_string", "sablock_version", "sablock_workspace_bytes",

@@ -9,6 +9,7 @@
 #include "stages.cuh"
 #include "score_simt.cuh"
 #include "score_tc.cuh"
+#include "score_fused.cuh"
 
 using namespace sab;
 
@@ -55,13 +56,15 @@ struct Plan {
     Geo geo;
     int n_prob, max_L;
     bool use_tc;
+    bool use_fused;            // the persistent two-sweep kernel (Llama-shaped problems)
+    int fu_cpp, fu_groups;     // its CTAs per problem group and number of groups
     int tpc1, tpc2;            // tiles per CTA of the tensor-core passes
     int n_chunks;              // pass-1 partials per row
     int keep_words, long_cap, seg_tiles;
     // workspace offsets
-    size_t o_status, o_ticket, o_long_count, o_tile_state, o_keep, control_bytes;
+    size_t o_status, o_ticket, o_long_count, o_tile_state, o_keep, o_arrive, o_done, control_bytes;
     size_t o_seg_id, o_seg_start, o_n_seg, o_s_raw, o_s, o_e, o_sr, o_part, o_lse, o_thr, o_cut, o_long_list,
-        o_phi, o_rank, total;
+        o_phi, o_rank, o_fpart, total;
 };
 
 bool tc_eligible(const sablock_params_t* p)
@@ -74,6 +77,35 @@ bool tc_eligible(const sablock_params_t* p)
     return true;
 }
 
+// The persistent kernel takes the shape whose 128 window rows per KV head fill one MMA tile.
+bool fused_eligible(const sablock_params_t* p)
+{
+    return tc_eligible(p) && p->head_dim == 128 && p->window == 32 && p->n_q_heads / p->n_kv_heads == 4;
+}
+
+constexpr int kFuMaxCtas = 256;       // upper bound on the CTAs of the persistent kernel (workspace sizing)
+
+// CTAs the persistent kernel may use on the current device: one per SM, all co-resident.
+int fused_cta_limit()
+{
+    static int cached[64];
+    static bool have[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    if (!have[dev]) {
+        int sms = 0, per_sm = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+        if (cudaFuncSetAttribute(score_fused_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kFuSmemBytes) != cudaSuccess ||
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, score_fused_tc, kFuThreads, kFuSmemBytes) != cudaSuccess) {
+            cudaGetLastError();
+            return 0;
+        }
+        cached[dev] = per_sm >= 1 ? (sms < kFuMaxCtas ? sms : kFuMaxCtas) : 0;
+        have[dev] = true;
+    }
+    return cached[dev];
+}
+
 sablock_status_t validate_params(const sablock_params_t* p)
 {
     if (!p) return SABLOCK_ERR_INVALID_ARG;
@@ -82,7 +114,7 @@ sablock_status_t validate_params(const sablock_params_t* p)
     if (p->dtype != SABLOCK_F32 && p->dtype != SABLOCK_BF16) return SABLOCK_ERR_INVALID_ARG;
     if (p->pool_kernel < 1 || (p->pool_kernel & 1) == 0) return SABLOCK_ERR_INVALID_ARG;
     if (p->pool_mode != 0 && p->pool_mode != 1) return SABLOCK_ERR_INVALID_ARG;
-    if (p->score_impl < 0 || p->score_impl > 2) return SABLOCK_ERR_INVALID_ARG;
+    if (p->score_impl < 0 || p->score_impl > 3) return SABLOCK_ERR_INVALID_ARG;
     if (!(p->tau >= 0.f) || !(p->alpha >= 0.f) || !(p->eta >= 0.f) || !(p->eps >= 0.f)) return SABLOCK_ERR_INVALID_ARG;
     if (p->k_stride_token < 0 || p->k_stride_head < 0 || p->k_stride_layer < 0 || p->v_stride_token < 0 ||
         p->v_stride_head < 0 || p->v_stride_layer < 0)
@@ -92,6 +124,7 @@ sablock_status_t validate_params(const sablock_params_t* p)
     const int es = p->dtype == SABLOCK_BF16 ? 2 : 4;
     if ((p->head_dim * es) % 16) return SABLOCK_ERR_UNSUPPORTED;
     if (p->score_impl == SABLOCK_SCORE_TENSOR && !tc_eligible(p)) return SABLOCK_ERR_UNSUPPORTED;
+    if (p->score_impl == SABLOCK_SCORE_FUSED && !fused_eligible(p)) return SABLOCK_ERR_UNSUPPORTED;
     return SABLOCK_OK;
 }
 
@@ -137,9 +170,10 @@ sablock_status_t make_plan(const sablock_params_t* p, int n_layers, int n_seqs, 
     pl->max_L = max_L;
     // The TMA boxes are 128 rows tall: tensors with fewer rows go to the SIMT kernels.
     const bool tc_rows_ok = total_tokens >= kTcTile && (long long)n_layers * n_seqs * g.H * g.window >= kTcTile;
-    pl->use_tc = p->score_impl == SABLOCK_SCORE_TENSOR ||
+    pl->use_tc = p->score_impl == SABLOCK_SCORE_TENSOR || p->score_impl == SABLOCK_SCORE_FUSED ||
                  (p->score_impl == SABLOCK_SCORE_AUTO && tc_eligible(p) && tc_rows_ok);
     const long long tiles = (max_L + kTcTile - 1) / kTcTile;
+    pl->use_fused = pl->use_tc && p->score_impl != SABLOCK_SCORE_TENSOR && fused_eligible(p);
     if (pl->use_tc) {
         long long work1 = tiles * g.Hkv * pl->n_prob, work2 = tiles * pl->n_prob;
         pl->tpc1 = (int)fmin(8.0, fmax(1.0, (double)(work1 / (148 * 4))));
@@ -160,6 +194,8 @@ sablock_status_t make_plan(const sablock_params_t* p, int n_layers, int n_seqs, 
     pl->o_long_count = take(sizeof(int) * pl->n_prob);
     pl->o_tile_state = take(sizeof(unsigned long long) * (size_t)n_seqs * pl->seg_tiles);
     pl->o_keep = take(sizeof(unsigned) * (size_t)pl->n_prob * pl->keep_words);
+    pl->o_arrive = take(sizeof(int) * (size_t)pl->n_prob * g.Hkv);
+    pl->o_done = take(sizeof(int) * (size_t)pl->n_prob * g.Hkv);
     pl->control_bytes = o;
     const size_t ntok = (size_t)n_layers * total_tokens;
     pl->o_seg_id = take(sizeof(int) * total_tokens);
@@ -178,6 +214,7 @@ sablock_status_t make_plan(const sablock_params_t* p, int n_layers, int n_seqs, 
     pl->o_long_list = take(sizeof(int) * (size_t)pl->n_prob * pl->long_cap);
     pl->o_phi = take(sizeof(double) * ntok);
     pl->o_rank = take(sizeof(int) * ntok);
+    pl->o_fpart = take(pl->use_fused ? sizeof(float2) * (size_t)kFuMaxCtas * kFuPartSlots * 2 * 128 : 0);
     pl->total = o;
     return SABLOCK_OK;
 }
@@ -292,6 +329,36 @@ sablock_status_t run_score(const Plan& pl, const sablock_params_t* p, const void
     if (pl.use_tc) {
         CUtensorMap tmQ, tmK;
         SAB_TRY(make_tensor_maps(pl, p, q, k, &tmQ, &tmK));
+        // Persistent two-sweep kernel: groups of CTAs each walk their share of the problems.
+        const int tiles_max = (pl.max_L + kTcTile - 1) / kTcTile;
+        const int min_cpp = (tiles_max + kFuMaxTilesPerCta - 1) / kFuMaxTilesPerCta;
+        const int n_cta = pl.use_fused ? fused_cta_limit() : 0;
+        if (pl.use_fused && n_cta >= min_cpp) {
+            int groups = n_cta / min_cpp;
+            if (groups > pl.n_prob) groups = pl.n_prob;
+            int cpp = n_cta / groups;
+            if (cpp > tiles_max) cpp = tiles_max;
+            FusedArgs fa;
+            fa.cpp = cpp; fa.n_groups = groups; fa.n_prob = pl.n_prob;
+            fa.c2 = c2; fa.eps = p->eps;
+            fa.part = at<float2>(ws, pl.o_fpart);
+            fa.lse2 = sb.lse2;
+            fa.arrive = at<int>(ws, pl.o_arrive);
+            fa.done = at<int>(ws, pl.o_done);
+            fa.s_out = s; fa.e_out = e; fa.status = status;
+            Geo geo = g;
+            void* args[] = {&tmQ, &tmK, &geo, &fa};
+            if (cudaLaunchCooperativeKernel((const void*)score_fused_tc, dim3(groups * cpp), dim3(kFuThreads), args,
+                                            kFuSmemBytes, stream) != cudaSuccess) {
+                cudaGetLastError();
+                return SABLOCK_ERR_CUDA;
+            }
+            ++t_launches;
+            prof_mark(1, stream);
+            prof_mark(2, stream);
+            return SABLOCK_OK;
+        }
+        if (p->score_impl == SABLOCK_SCORE_FUSED) return SABLOCK_ERR_UNSUPPORTED;
         constexpr int NST1 = 2;
         const int n_atoms = g.D / 64;
         const int smem1 = 1024 + (1 + NST1) * n_atoms * kAtomBytes;
