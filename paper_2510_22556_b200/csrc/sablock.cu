@@ -83,7 +83,7 @@ bool fused_eligible(const sablock_params_t* p)
     return tc_eligible(p) && p->head_dim == 128 && p->window == 32 && p->n_q_heads / p->n_kv_heads == 4;
 }
 
-constexpr int kFuMaxCtas = 256;       // upper bound on the CTAs of the persistent kernel (workspace sizing)
+constexpr int kFuMaxCtas = kFuMaxCtasDev;   // upper bound on the CTAs of the persistent kernel (workspace sizing)
 
 // CTAs the persistent kernel may use on the current device: one per SM, all co-resident.
 int fused_cta_limit()
@@ -767,5 +767,13 @@ sablock_status_t sablock_compress_layers_host(const sablock_params_t* p, int n_l
         return SABLOCK_ERR_CUDA;
     return cudaStreamSynchronize(st) == cudaSuccess ? SABLOCK_OK : SABLOCK_ERR_CUDA;
 }
+
+#ifdef SABLOCK_TRACE
+/* Trace builds only: copies the cycle stamps of the traced CTAs to host memory. */
+int sablock_trace_dump(long long* out)
+{
+    return (int)cudaMemcpyFromSymbol(out, sab::g_trace, sizeof(sab::g_trace));
+}
+#endif
 
 }  // extern "C"

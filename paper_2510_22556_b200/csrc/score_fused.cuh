@@ -37,8 +37,9 @@ constexpr int kFuStages = 4;                 // K tile ring
 constexpr int kFuMaxTilesPerCta = 7;         // \bar A slots in tensor memory: 7 x 32 columns
 constexpr int kFuAbarCol0 = 256;             // columns [0, 256): two logit accumulators
 constexpr int kFuTmemCols = 512;
-constexpr int kFuLead = 2;                   // sweep A runs this many tiles ahead of sweep B
+constexpr int kFuLead = 3;                   // sweep A runs this many tiles ahead of sweep B
 constexpr int kFuPartSlots = 4;              // ring of per-phase partial buffers
+constexpr int kFuMaxCtasDev = 256;           // upper bound on the CTAs of one launch
 constexpr int kFuTileBytes = 2 * kAtomBytes; // 128 rows x 128 bf16
 constexpr int kFuSmemBytes = 1024 + (2 + kFuStages) * kFuTileBytes;
 
@@ -57,6 +58,19 @@ struct FusedArgs {
     int* status;
 };
 
+// Optional cycle-stamp trace of a few CTAs (compiled in with -DSABLOCK_TRACE; off otherwise):
+// role 0 = TMA producer, 1 = MMA issuer, 2 / 3 = leader thread of epilogue set 0 / 1.
+#ifdef SABLOCK_TRACE
+constexpr int kTraceOps = 600;
+__device__ long long g_trace[4][4][kTraceOps][4];   // [traced CTA][role][op][event]
+#define FU_TRACE(role, n, ev)                                                                 \
+    do {                                                                                      \
+        if (tslot >= 0 && (n) < kTraceOps) g_trace[tslot][role][n][ev] = clock64();           \
+    } while (0)
+#else
+#define FU_TRACE(role, n, ev) do { } while (0)
+#endif
+
 struct FuBarriers {
     uint64_t full[kFuStages];
     uint64_t empty[kFuStages];
@@ -64,77 +78,93 @@ struct FuBarriers {
     uint64_t tempty[2];
     uint64_t qfull[2];
     uint64_t qempty[2];
-    uint64_t ebar;           // all epilogue threads
-    uint64_t pbar[4];        // the two warps of one tensor-memory lane quarter
+    uint64_t sbar[2];        // the four warps of one epilogue set
     uint32_t tmem_base;
     int abort_flag;
 };
 
 // One step of a CTA's work list.
 enum { kOpA = 0, kOpB = 1, kOpPairEnd = 2, kOpStop = 3 };
+
+// What a role needs to know about one phase = (problem, KV head).
+struct FuPhase {
+    int phase;       // phase counter of the group; -1 = none
+    int prob, j;     // problem index and KV head
+    int layer, seq;
+    int L, Tn;       // sequence length and compressible length
+    int tok_base;    // first packed token row of the sequence
+    int n_tiles;     // tiles of this CTA in the sweep in question
+};
+
 struct FuOp {
     int kind;
-    int phase;       // phase counter of the group (problem slot * Hkv + KV head)
-    int prob, j;     // problem index and KV head of that phase
     int k;           // which of the CTA's tiles (slot of \bar A in tensor memory)
     int tile;        // token tile index inside the sequence
-    int first, last; // first / last tile of this kind for this CTA in this phase
+    int last;        // last tile of this kind for this CTA in this phase
     int pair;        // for kOpPairEnd: the pair that ended
 };
 
-// Deterministic walk over the work list; every role of the CTA runs its own copy.
+// Deterministic walk over the work list; every role of the CTA runs its own copy.  Pair n holds
+// the sweep A tiles of phase n (`pa`) and the sweep B tiles of phase n - 1 (`pb`); all divisions
+// happen when a pair begins, the per-tile step is a few adds and compares.
 struct FuIter {
     const Geo& g;
-    int cpp, n_groups, n_prob, group, rank;
+    int cpp, n_groups, group, rank;
     int n_phases;            // phases of this group
-    int pair, ia, ib, nA, nB;
-    __device__ FuIter(const Geo& geo, const FusedArgs& a)
-        : g(geo), cpp(a.cpp), n_groups(a.n_groups), n_prob(a.n_prob)
+    int pair, ia, ib;
+    FuPhase pa, pb;
+    __device__ FuIter(const Geo& geo, const FusedArgs& a) : g(geo), cpp(a.cpp), n_groups(a.n_groups)
     {
         group = blockIdx.x / cpp;
         rank = blockIdx.x % cpp;
-        const int my_probs = group < n_groups ? (n_prob - group + n_groups - 1) / n_groups : 0;
+        const int my_probs = group < n_groups ? (a.n_prob - group + n_groups - 1) / n_groups : 0;
         n_phases = my_probs * g.Hkv;
         pair = 0; ia = ib = 0;
-        load_pair();
+        pb.phase = -1; pb.n_tiles = 0;
+        load_a();
     }
-    __device__ int prob_of(int phase) const { return group + (phase / g.Hkv) * n_groups; }
-    __device__ int tiles_of(int phase, bool sweep_b) const
+    __device__ int my_tiles(int n) const { return rank < n ? (n - rank + cpp - 1) / cpp : 0; }
+    __device__ void load_a()
     {
-        if (phase < 0 || phase >= n_phases) return 0;
-        const int seq = prob_of(phase) % g.n_seqs;
-        if (geo_identity(g, seq)) return 0;
-        const int L = geo_L(g, seq);
-        const int n = sweep_b ? (L - g.window + kTcTile - 1) / kTcTile : (L + kTcTile - 1) / kTcTile;
-        return rank < n ? (n - rank + cpp - 1) / cpp : 0;
+        pa.phase = pair;
+        pa.n_tiles = 0;
+        if (pair >= n_phases) { pa.phase = -1; return; }
+        pa.prob = group + (pair / g.Hkv) * n_groups;
+        pa.j = pair % g.Hkv;
+        pa.layer = pa.prob / g.n_seqs;
+        pa.seq = pa.prob % g.n_seqs;
+        pa.tok_base = g.cu[pa.seq];
+        pa.L = g.cu[pa.seq + 1] - pa.tok_base;
+        pa.Tn = pa.L - g.window;
+        if (pa.L > g.n_out) pa.n_tiles = my_tiles((pa.L + kTcTile - 1) / kTcTile);   // else: returned unchanged
     }
-    __device__ void load_pair()
+    __device__ void next_pair()
     {
-        nA = tiles_of(pair, false);
-        nB = tiles_of(pair - 1, true);
+        pb = pa;
+        pb.n_tiles = (pa.phase >= 0 && pa.L > g.n_out) ? my_tiles((pa.Tn + kTcTile - 1) / kTcTile) : 0;
+        ++pair; ia = ib = 0;
+        load_a();
     }
     __device__ FuOp next()
     {
         FuOp op;
         op.pair = pair;
         if (pair > n_phases) { op.kind = kOpStop; return op; }
-        const bool take_a = ia < nA && (ia < ib + kFuLead || ib >= nB);
-        if (take_a || ib < nB) {
-            op.kind = take_a ? kOpA : kOpB;
-            op.phase = take_a ? pair : pair - 1;
-            op.k = take_a ? ia : ib;
-            const int n = take_a ? nA : nB;
-            op.first = op.k == 0;
-            op.last = op.k == n - 1;
-            op.tile = rank + op.k * cpp;
-            op.prob = prob_of(op.phase);
-            op.j = op.phase % g.Hkv;
-            if (take_a) ++ia; else ++ib;
+        const bool take_a = ia < pa.n_tiles && (ia < ib + kFuLead || ib >= pb.n_tiles);
+        if (take_a) {
+            op.kind = kOpA; op.k = ia; op.last = ia == pa.n_tiles - 1;
+            op.tile = rank + ia * cpp;
+            ++ia;
+            return op;
+        }
+        if (ib < pb.n_tiles) {
+            op.kind = kOpB; op.k = ib; op.last = ib == pb.n_tiles - 1;
+            op.tile = rank + ib * cpp;
+            ++ib;
             return op;
         }
         op.kind = kOpPairEnd;
-        ++pair; ia = ib = 0;
-        load_pair();
+        next_pair();
         return op;
     }
 };
@@ -195,6 +225,25 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const float (&v)[16])
           "r"(__float_as_uint(v[15]))
         : "memory");
 }
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
+          "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])),
+          "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])),
+          "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
+          "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])),
+          "r"(__float_as_uint(v[15])), "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])),
+          "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])), "r"(__float_as_uint(v[20])),
+          "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])),
+          "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])),
+          "r"(__float_as_uint(v[27])), "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])),
+          "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
+        : "memory");
+}
 __device__ __forceinline__ void tmem_st_wait()
 {
     asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
@@ -243,6 +292,61 @@ __device__ __forceinline__ float chunk_max(const uint32_t (&r)[32])
     }
     return fmaxf(a, b);
 }
+// Causal mask of 32 logits of window row w: keys beyond position lim = T + w do not exist for it.
+__device__ __forceinline__ void chunk_mask(uint32_t (&r)[32], int tok0, int lim)
+{
+#pragma unroll
+    for (int i = 0; i < 32; ++i)
+        if (tok0 + i > lim) r[i] = 0xff800000u;       // -inf
+}
+
+// Running sum of exp2 over the keys of one window row, kept as l * 2^m with an integer-valued
+// reference exponent m that only moves when the sum would leave the fp32 range.
+struct RowSum {
+    float m, l;
+    bool have_m;
+    __device__ void reset() { m = 0.f; l = 0.f; have_m = false; }
+    __device__ void add(const uint32_t (&r0)[32], const uint32_t (&r1)[32], float c2)
+    {
+        if (!have_m) {
+            const float mx = fmaxf(chunk_max(r0), chunk_max(r1)) * c2;
+            m = (mx == -INFINITY) ? 0.f : ceilf(mx);
+            have_m = true;
+        }
+        float c = chunk_expsum(r0, c2, m) + chunk_expsum(r1, c2, m);
+        if (!(l + c < 1.8e19f)) {                          // far above the reference: move it
+            const float mx = fmaxf(chunk_max(r0), chunk_max(r1)) * c2;
+            const float m_new = fmaxf(m, ceilf(mx));
+            l *= exp2f(m - m_new);
+            m = m_new;
+            c = chunk_expsum(r0, c2, m) + chunk_expsum(r1, c2, m);
+        }
+        l += c;
+    }
+};
+
+// accw[w] += exp2(logit * c2 - lse) for two heads' 32 window positions each (64 logits).
+__device__ __forceinline__ void accumulate_heads(float (&accw)[32], const uint32_t (&r0)[32], const uint32_t (&r1)[32],
+                                                 const float* lse0, float c2)
+{
+    const float4* l4 = reinterpret_cast<const float4*>(lse0);
+#pragma unroll
+    for (int i = 0; i < 32; i += 4) {
+        const float4 ls = l4[i >> 2];
+        accw[i + 0] += ex2_approx(fmaf(__uint_as_float(r0[i + 0]), c2, -ls.x));
+        accw[i + 1] += ex2_approx(fmaf(__uint_as_float(r0[i + 1]), c2, -ls.y));
+        accw[i + 2] += ex2_approx(fmaf(__uint_as_float(r0[i + 2]), c2, -ls.z));
+        accw[i + 3] += ex2_approx(fmaf(__uint_as_float(r0[i + 3]), c2, -ls.w));
+    }
+#pragma unroll
+    for (int i = 0; i < 32; i += 4) {
+        const float4 ls = l4[8 + (i >> 2)];
+        accw[i + 0] += ex2_approx(fmaf(__uint_as_float(r1[i + 0]), c2, -ls.x));
+        accw[i + 1] += ex2_approx(fmaf(__uint_as_float(r1[i + 1]), c2, -ls.y));
+        accw[i + 2] += ex2_approx(fmaf(__uint_as_float(r1[i + 2]), c2, -ls.z));
+        accw[i + 3] += ex2_approx(fmaf(__uint_as_float(r1[i + 3]), c2, -ls.w));
+    }
+}
 
 __global__ void __launch_bounds__(kFuThreads, 1)
 score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const Geo g,
@@ -250,8 +354,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 {
     extern __shared__ uint8_t dyn_smem[];
     __shared__ FuBarriers sh;
-    __shared__ __align__(16) float lse_s[2][128];
-    __shared__ float xch[2][2][2][128];          // [op parity][tot | ent][half][token row]
+    __shared__ __align__(16) float lse_s[2][2][128];     // [epilogue set][phase parity][window row]
     const uint32_t base = (smem_u32(dyn_smem) + 1023u) & ~1023u;
     const uint32_t q_smem = base;                                  // two query blocks
     const uint32_t k_smem = base + 2 * kFuTileBytes;               // K tile ring
@@ -264,12 +367,11 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&sh.tfull[i]), 1);
-            mbar_init(smem_u32(&sh.tempty[i]), kFuEpiThreads);
+            mbar_init(smem_u32(&sh.tempty[i]), 128);
             mbar_init(smem_u32(&sh.qfull[i]), 1);
             mbar_init(smem_u32(&sh.qempty[i]), 1);
+            mbar_init(smem_u32(&sh.sbar[i]), 128);
         }
-        mbar_init(smem_u32(&sh.ebar), kFuEpiThreads);
-        for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&sh.pbar[i]), 64);
         sh.abort_flag = 0;
         fence_mbar_init();
     }
@@ -283,7 +385,10 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     tc_fence_after();
     const uint32_t tmem = sh.tmem_base;
     volatile int* abort_flag = &sh.abort_flag;
-    const int R = 128;                               // window rows per KV head
+    constexpr int R = 128;                           // window rows per KV head
+#ifdef SABLOCK_TRACE
+    const int tslot = blockIdx.x == 0 ? 0 : blockIdx.x == 5 ? 1 : blockIdx.x == 77 ? 2 : blockIdx.x == gridDim.x - 1 ? 3 : -1;
+#endif
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -295,28 +400,29 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             const uint64_t pol_q = l2_policy_evict_last();
             FuIter it(g, fa);
             int n_ops = 0, qloads[2] = {0, 0}, q_phase = -1;
-            bool ok = true;
-            while (ok) {
+            while (true) {
                 const FuOp op = it.next();
                 if (op.kind == kOpStop) break;
                 if (op.kind == kOpPairEnd) continue;
-                if (op.kind == kOpA && op.phase != q_phase) {      // first tile of a phase: its query block
-                    q_phase = op.phase;
-                    const int b = op.phase & 1;
+                const FuPhase& ph = op.kind == kOpA ? it.pa : it.pb;
+                if (op.kind == kOpA && ph.phase != q_phase) {      // first tile of a phase: its query block
+                    q_phase = ph.phase;
+                    const int b = ph.phase & 1;
                     if (qloads[b] > 0 && !mbar_wait(smem_u32(&sh.qempty[b]), (qloads[b] - 1) & 1, abort_flag)) break;
                     ++qloads[b];
                     mbar_expect_tx(smem_u32(&sh.qfull[b]), kFuTileBytes);
                     for (int a = 0; a < 2; ++a)
                         tma_load_2d(q_smem + b * kFuTileBytes + a * kAtomBytes, &tmQ, smem_u32(&sh.qfull[b]), a * 64,
-                                    op.prob * g.H * g.window + op.j * R, pol_q);
+                                    ph.prob * g.H * g.window + ph.j * R, pol_q);
                 }
-                const int st = n_ops % kFuStages, ph = (n_ops / kFuStages) & 1;
-                if (!mbar_wait(smem_u32(&sh.empty[st]), ph ^ 1, abort_flag)) break;
+                const int st = n_ops % kFuStages, par = (n_ops / kFuStages) & 1;
+                FU_TRACE(0, n_ops, 0);
+                if (!mbar_wait(smem_u32(&sh.empty[st]), par ^ 1, abort_flag)) break;
+                FU_TRACE(0, n_ops, 1);
                 mbar_expect_tx(smem_u32(&sh.full[st]), kFuTileBytes);
-                const int layer = op.prob / g.n_seqs, seq = op.prob % g.n_seqs;
                 for (int a = 0; a < 2; ++a)
-                    tma_load_4d(k_smem + st * kFuTileBytes + a * kAtomBytes, &tmK, smem_u32(&sh.full[st]), a * 64, op.j,
-                                g.cu[seq] + op.tile * kTcTile, layer, op.kind == kOpA ? pol_a : pol_b);
+                    tma_load_4d(k_smem + st * kFuTileBytes + a * kAtomBytes, &tmK, smem_u32(&sh.full[st]), a * 64, ph.j,
+                                ph.tok_base + op.tile * kTcTile, ph.layer, op.kind == kOpA ? pol_a : pol_b);
                 ++n_ops;
             }
         }
@@ -338,17 +444,21 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     }
                     continue;
                 }
-                const int b = op.phase & 1;
-                if (op.kind == kOpA && op.phase != q_phase) {
-                    q_phase = op.phase;
+                const FuPhase& ph = op.kind == kOpA ? it.pa : it.pb;
+                const int b = ph.phase & 1;
+                if (op.kind == kOpA && ph.phase != q_phase) {
+                    q_phase = ph.phase;
                     if (!mbar_wait(smem_u32(&sh.qfull[b]), qwaits[b] & 1, abort_flag)) break;
                     ++qwaits[b];
                     q_used[b] = true;
                 }
-                const int st = n_ops % kFuStages, ph = (n_ops / kFuStages) & 1;
+                const int st = n_ops % kFuStages, par = (n_ops / kFuStages) & 1;
                 const int acc = n_ops & 1, aph = (n_ops >> 1) & 1;
+                FU_TRACE(1, n_ops, 0);
                 if (!mbar_wait(smem_u32(&sh.tempty[acc]), aph ^ 1, abort_flag)) break;
-                if (!mbar_wait(smem_u32(&sh.full[st]), ph, abort_flag)) break;
+                FU_TRACE(1, n_ops, 1);
+                if (!mbar_wait(smem_u32(&sh.full[st]), par, abort_flag)) break;
+                FU_TRACE(1, n_ops, 2);
                 tc_fence_after();
                 const uint32_t kt = k_smem + st * kFuTileBytes, qt = q_smem + b * kFuTileBytes;
                 if (op.kind == kOpA) tc_issue_tile(tmem, acc, qt, kt, 8);     // rows = window rows
@@ -363,10 +473,10 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         FuIter it(g, fa);
         const int group = it.group, rank = it.rank;
         for (int phase = 0; phase < it.n_phases; ++phase) {
-            const int prob = it.prob_of(phase), j = phase % g.Hkv, seq = prob % g.n_seqs;
+            const int prob = group + (phase / g.Hkv) * fa.n_groups, j = phase % g.Hkv, seq = prob % g.n_seqs;
             if (geo_identity(g, seq)) continue;
             const int nt1 = (geo_L(g, seq) + kTcTile - 1) / kTcTile;
-            const int n_src = min(fa.cpp, nt1);                 // CTAs that hold tiles of this problem
+            const int n_src = 2 * min(fa.cpp, nt1);             // (CTA that holds tiles, epilogue set)
             if (rank >= R) continue;
             bool ok = true;
             if (lane == 0) ok = wait_counter(fa.arrive + prob * g.Hkv + j, n_src, abort_flag, fa.status);
@@ -374,19 +484,25 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             if (!ok) break;
             const float2* pp = fa.part + ((size_t)group * kFuPartSlots + (phase % kFuPartSlots)) * fa.cpp * 2 * R;
             for (int row = rank; row < R; row += fa.cpp) {
-                // partial i = (source CTA, column half); merged in index order
-                float m = -INFINITY;
-                for (int i = lane; i < 2 * n_src; i += 32) {
-                    const float2 v = __ldcg(pp + (size_t)i * R + row);
-                    if (v.y > 0.f) m = fmaxf(m, v.x);
+                // partial i = (source CTA, epilogue set), merged in index order; all loads of a
+                // lane are issued before the first use so that their latencies overlap
+                constexpr int kPer = 2 * kFuMaxCtasDev / 32;
+                float2 v[kPer];
+#pragma unroll
+                for (int u = 0; u < kPer; ++u) {
+                    const int i = lane + 32 * u;
+                    v[u] = i < n_src ? __ldcg(pp + (size_t)i * R + row) : make_float2(0.f, 0.f);
                 }
+                float m = -INFINITY;
+#pragma unroll
+                for (int u = 0; u < kPer; ++u)
+                    if (v[u].y > 0.f) m = fmaxf(m, v[u].x);
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
                 float l = 0.f;
-                for (int i = lane; i < 2 * n_src; i += 32) {
-                    const float2 v = __ldcg(pp + (size_t)i * R + row);
-                    if (v.y > 0.f) l += v.y * exp2f(v.x - m);
-                }
+#pragma unroll
+                for (int u = 0; u < kPer; ++u)
+                    if (v[u].y > 0.f) l += v[u].y * exp2f(v[u].x - m);
                 l = warp_sum(l);
                 if (lane == 0) fa.lse2[(size_t)prob * g.H * g.window + j * R + row] = m + log2f(l);
             }
@@ -398,150 +514,142 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         }
     } else if (warp >= kFuEpiWarp0 && warp < kFuEpiWarp0 + 8) {
         // ------------------------------------------------------------------ epilogue
+        // Two sets of four warps; set s takes the tiles whose logits land in accumulator s, so
+        // the sets run half a tile out of step and one computes while the other waits and loads.
         const int ew = warp - kFuEpiWarp0;
         const int q4 = warp & 3;                       // tensor-memory lane quarter of this warp
-        const int half = ew >> 2;                      // which half of the columns / window positions
+        const int set = ew >> 2;
         const int row = q4 * 32 + lane;                // TMEM lane: window row (sweep A) or token (sweep B)
-        const int et = ew * 32 + lane;                 // thread index among the epilogue threads
+        const bool leader = (ew & 3) == 0 && lane == 0;
         const uint32_t lane_addr = tmem + ((uint32_t)(q4 * 32) << 16);
+        const uint32_t acc_addr = lane_addr + (uint32_t)set * 128u;
         const float c2 = fa.c2;
         const float inv_H = 1.f / (float)g.H;
+        const int n_mergers = min(fa.cpp, R);
         FuIter it(g, fa);
         const int group = it.group, rank = it.rank;
-        float m_ref = 0.f, l_run = 0.f;                // sweep A state of (row, half)
-        bool have_m = false;
-        int n_ops = 0, n_fin = 0, lse_phase = -1, n_esync = 0, n_psync = 0;
+        RowSum rs;                                     // sweep A state of this window row in this set
+        rs.reset();
+        int n_ops = 0, n_mine = 0, lse_phase = -1, n_sync = 0;
         while (true) {
             const FuOp op = it.next();
             if (op.kind == kOpStop) break;
             if (op.kind == kOpPairEnd) continue;
-            const int seq = op.prob % g.n_seqs, layer = op.prob / g.n_seqs;
-            const int L = geo_L(g, seq), Tn = L - g.window;
-            const int acc = n_ops & 1, aph = (n_ops >> 1) & 1;
-            const uint32_t acc_addr = lane_addr + (uint32_t)acc * 128u;
+            const bool mine = (n_ops & 1) == set;
+            ++n_ops;
             if (op.kind == kOpA) {
-                if (op.first) { have_m = false; m_ref = 0.f; l_run = 0.f; }
-                if (!mbar_wait(smem_u32(&sh.tfull[acc]), aph, abort_flag)) break;
-                tc_fence_after();
-                const int tok0 = op.tile * kTcTile + half * 64;
-                const int lim = Tn + (row & 31);                   // causal: key index <= T + w (Eq. 2)
-                const bool need_mask = tok0 + 63 > Tn;
-                uint32_t r0[32], r1[32];
-                tmem_ld32_issue(acc_addr + half * 64, r0);
-                tmem_ld32_issue(acc_addr + half * 64 + 32, r1);
-                tmem_ld_wait();
-                tc_fence_before();
-                mbar_arrive(smem_u32(&sh.tempty[acc]));            // logits are in registers: release the accumulator
-                if (need_mask) {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        if (tok0 + i > lim) r0[i] = 0xff800000u;       // -inf
-                        if (tok0 + 32 + i > lim) r1[i] = 0xff800000u;
-                    }
+                const FuPhase& ph = it.pa;
+                if (mine) {
+                    if (leader) FU_TRACE(2 + set, n_mine, 0);
+                    if (!mbar_wait(smem_u32(&sh.tfull[set]), n_mine & 1, abort_flag)) break;
+                    if (leader) FU_TRACE(2 + set, n_mine, 1);
+                    tc_fence_after();
+                    const int tok0 = op.tile * kTcTile;
+                    const int lim = ph.Tn + (row & 31);            // causal: key index <= T + w (Eq. 2)
+                    const bool need_mask = tok0 + 127 > ph.Tn;
+                    uint32_t r0[32], r1[32];
+                    tmem_ld32_issue(acc_addr, r0);
+                    tmem_ld32_issue(acc_addr + 32, r1);
+                    tmem_ld_wait();
+                    if (need_mask) { chunk_mask(r0, tok0, lim); chunk_mask(r1, tok0 + 32, lim); }
+                    rs.add(r0, r1, c2);
+                    tmem_ld32_issue(acc_addr + 64, r0);
+                    tmem_ld32_issue(acc_addr + 96, r1);
+                    tmem_ld_wait();
+                    tc_fence_before();
+                    mbar_arrive(smem_u32(&sh.tempty[set]));        // logits are in registers: release the accumulator
+                    if (leader) FU_TRACE(2 + set, n_mine, 2);
+                    if (need_mask) { chunk_mask(r0, tok0 + 64, lim); chunk_mask(r1, tok0 + 96, lim); }
+                    rs.add(r0, r1, c2);
+                    if (leader) FU_TRACE(2 + set, n_mine, 3);
+                    ++n_mine;
                 }
-                if (!have_m) {                                     // reference exponent of this row
-                    const float mx = fmaxf(chunk_max(r0), chunk_max(r1)) * c2;
-                    m_ref = (mx == -INFINITY) ? 0.f : ceilf(mx);
-                    have_m = true;
-                }
-                float c = chunk_expsum(r0, c2, m_ref) + chunk_expsum(r1, c2, m_ref);
-                if (!(l_run + c < 1.8e19f)) {                      // far above the reference: move it
-                    const float mx = fmaxf(chunk_max(r0), chunk_max(r1)) * c2;
-                    const float m_new = fmaxf(m_ref, ceilf(mx));
-                    l_run *= exp2f(m_ref - m_new);
-                    m_ref = m_new;
-                    c = chunk_expsum(r0, c2, m_ref) + chunk_expsum(r1, c2, m_ref);
-                }
-                l_run += c;
                 if (op.last) {
-                    // The partial buffers are a ring over phases: the slot is free once every merge
-                    // of the phase that used it last is done.  (A CTA that also runs sweep B is
-                    // throttled by it anyway; one that owns only a window tile is not.)
-                    if (et == 0 && op.phase >= kFuPartSlots) {
-                        const int old = op.phase - kFuPartSlots;
-                        wait_counter(fa.done + it.prob_of(old) * g.Hkv + old % g.Hkv, min(fa.cpp, R), abort_flag, fa.status);
+                    // Publish this set's row sums of the phase.  The partial buffers are a ring over
+                    // phases: the slot is free once every merge of the phase that used it last is
+                    // done.  (A CTA that also runs sweep B is throttled by it anyway; one that owns
+                    // only a window tile is not.)
+                    if (leader && ph.phase >= kFuPartSlots) {
+                        const int old = ph.phase - kFuPartSlots;
+                        wait_counter(fa.done + (group + (old / g.Hkv) * fa.n_groups) * g.Hkv + old % g.Hkv, n_mergers,
+                                     abort_flag, fa.status);
                     }
-                    if (!group_sync(&sh.ebar, n_esync, abort_flag)) break;
-                    float2* pp = fa.part + ((size_t)group * kFuPartSlots + (op.phase % kFuPartSlots)) * fa.cpp * 2 * R;
-                    pp[((size_t)rank * 2 + half) * R + row] = make_float2(m_ref, l_run);
+                    if (!group_sync(&sh.sbar[set], n_sync, abort_flag)) break;
+                    float2* pp = fa.part + ((size_t)group * kFuPartSlots + (ph.phase % kFuPartSlots)) * fa.cpp * 2 * R;
+                    pp[((size_t)rank * 2 + set) * R + row] = make_float2(rs.m, rs.l);
                     __threadfence();
-                    if (!group_sync(&sh.ebar, n_esync, abort_flag)) break;
-                    if (et == 0) atomicAdd(fa.arrive + op.prob * g.Hkv + op.j, 1);
+                    if (!group_sync(&sh.sbar[set], n_sync, abort_flag)) break;
+                    if (leader) atomicAdd(fa.arrive + ph.prob * g.Hkv + ph.j, 1);
+                    rs.reset();
                 }
-            } else {
-                if (op.phase != lse_phase) {                       // log-sum-exps of this phase
-                    lse_phase = op.phase;
-                    if (et == 0) wait_counter(fa.done + op.prob * g.Hkv + op.j, min(fa.cpp, R), abort_flag, fa.status);
-                    if (!group_sync(&sh.ebar, n_esync, abort_flag)) break;
-                    if (et < R) lse_s[op.phase & 1][et] = __ldcg(fa.lse2 + (size_t)op.prob * g.H * g.window + op.j * R + et);
-                    if (!group_sync(&sh.ebar, n_esync, abort_flag)) break;
+            } else if (mine) {
+                const FuPhase& ph = it.pb;
+                if (ph.phase != lse_phase) {                       // log-sum-exps of this phase
+                    lse_phase = ph.phase;
+                    if (leader) wait_counter(fa.done + ph.prob * g.Hkv + ph.j, n_mergers, abort_flag, fa.status);
+                    if (!group_sync(&sh.sbar[set], n_sync, abort_flag)) break;
+                    lse_s[set][ph.phase & 1][row] = __ldcg(fa.lse2 + (size_t)ph.prob * g.H * g.window + ph.j * R + row);
+                    if (!group_sync(&sh.sbar[set], n_sync, abort_flag)) break;
                 }
-                if (!mbar_wait(smem_u32(&sh.tfull[acc]), aph, abort_flag)) break;
+                if (leader) FU_TRACE(2 + set, n_mine, 0);
+                if (!mbar_wait(smem_u32(&sh.tfull[set]), n_mine & 1, abort_flag)) break;
+                if (leader) FU_TRACE(2 + set, n_mine, 1);
                 tc_fence_after();
-                uint32_t v[4][16];                                 // head hl of the group, 16 window positions
+                const float* lj = lse_s[set][ph.phase & 1];
+                float accw[32];
 #pragma unroll
-                for (int hl = 0; hl < 4; ++hl) tmem_ld16_issue(acc_addr + hl * 32 + half * 16, v[hl]);
+                for (int i = 0; i < 32; ++i) accw[i] = 0.f;
+                uint32_t r0[32], r1[32];
+                tmem_ld32_issue(acc_addr, r0);                     // query heads 0, 1 of the group
+                tmem_ld32_issue(acc_addr + 32, r1);
+                tmem_ld_wait();
+                accumulate_heads(accw, r0, r1, lj, c2);
+                tmem_ld32_issue(acc_addr + 64, r0);                // query heads 2, 3
+                tmem_ld32_issue(acc_addr + 96, r1);
                 tmem_ld_wait();
                 tc_fence_before();
-                mbar_arrive(smem_u32(&sh.tempty[acc]));
-                const float* lj = lse_s[op.phase & 1];
-                float accw[16];
-#pragma unroll
-                for (int i = 0; i < 16; ++i) accw[i] = 0.f;
-#pragma unroll
-                for (int hl = 0; hl < 4; ++hl) {
-                    const float4* l4 = reinterpret_cast<const float4*>(lj + hl * 32 + half * 16);
-#pragma unroll
-                    for (int i = 0; i < 16; i += 4) {
-                        const float4 ls = l4[i >> 2];
-                        accw[i + 0] += ex2_approx(fmaf(__uint_as_float(v[hl][i + 0]), c2, -ls.x));
-                        accw[i + 1] += ex2_approx(fmaf(__uint_as_float(v[hl][i + 1]), c2, -ls.y));
-                        accw[i + 2] += ex2_approx(fmaf(__uint_as_float(v[hl][i + 2]), c2, -ls.z));
-                        accw[i + 3] += ex2_approx(fmaf(__uint_as_float(v[hl][i + 3]), c2, -ls.w));
-                    }
-                }
+                mbar_arrive(smem_u32(&sh.tempty[set]));
+                if (leader) FU_TRACE(2 + set, n_mine, 2);
+                accumulate_heads(accw, r0, r1, lj + 64, c2);
+                const int n_this = n_mine;
+                ++n_mine;
                 // \bar A of this token tile, summed over the KV heads seen so far
-                const uint32_t abar_addr = lane_addr + (uint32_t)(kFuAbarCol0 + op.k * 32 + half * 16);
-                if (op.j > 0) {
-                    uint32_t prev[16];
-                    tmem_ld16_issue(abar_addr, prev);
+                const uint32_t abar_addr = lane_addr + (uint32_t)(kFuAbarCol0 + op.k * 32);
+                if (ph.j > 0) {
+                    tmem_ld32_issue(abar_addr, r0);
                     tmem_ld_wait();
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) accw[i] += __uint_as_float(prev[i]);
+                    for (int i = 0; i < 32; ++i) accw[i] += __uint_as_float(r0[i]);
                 }
-                if (op.j < g.Hkv - 1) {
-                    tmem_st16(abar_addr, accw);
+                if (ph.j < g.Hkv - 1) {
+                    tmem_st32(abar_addr, accw);
                     tmem_st_wait();
+                    tc_fence_before();         // the next head's update may come from the other set's warps
                 } else {
                     // last KV head of the layer: s_t (Eqs. 3, 4) and the entropy of Eq. 6
-                    const int par = n_fin & 1;
-                    ++n_fin;
-                    float tot_h = 0.f;
+                    float t0 = 0.f, t1 = 0.f, t2 = 0.f, t3 = 0.f;
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) tot_h += accw[i];
-                    xch[par][0][half][row] = tot_h;
-                    if (!group_sync(&sh.pbar[q4], n_psync, abort_flag)) break;
-                    const float tot = xch[par][0][0][row] + xch[par][0][1][row];
-                    float ent_h = 0.f;
+                    for (int i = 0; i < 32; i += 4) { t0 += accw[i]; t1 += accw[i + 1]; t2 += accw[i + 2]; t3 += accw[i + 3]; }
+                    const float tot = (t0 + t1) + (t2 + t3);
+                    float ent = 0.f;
                     if (tot > 0.f) {
                         const float inv = 1.f / tot;
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) {
+                        for (int i = 0; i < 32; ++i) {
                             const float ah = accw[i] * inv;                       // \hat A (Eq. 6)
-                            ent_h -= ah * (lg2_approx(ah + fa.eps) * 0.6931471805599453f);
+                            ent -= ah * (lg2_approx(ah + fa.eps) * 0.6931471805599453f);
                         }
                     }
-                    xch[par][1][half][row] = ent_h;
-                    if (!group_sync(&sh.pbar[q4], n_psync, abort_flag)) break;
                     const int t = op.tile * kTcTile + row;
-                    if (half == 0 && t < Tn) {
-                        const size_t off = (size_t)layer * g.total_tokens + g.cu[seq];
+                    if (t < ph.Tn) {
+                        const size_t off = (size_t)ph.layer * g.total_tokens + ph.tok_base;
                         fa.s_out[off + t] = tot * inv_H;
-                        fa.e_out[off + t] = xch[par][1][0][row] + xch[par][1][1][row];
+                        fa.e_out[off + t] = ent;
                     }
                 }
+                if (leader) FU_TRACE(2 + set, n_this, 3);
+                (void)n_this;
             }
-            ++n_ops;
         }
     }
 
