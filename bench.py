@@ -194,6 +194,9 @@ def run_ours(args):
     ab = algorithmic_bytes(cfg, nl, total, out.n_out)
     dom = max(("score_pass1", "score_pass2"), key=lambda k: stage_avg.get(k, 0.0))
     dom_ms = stage_avg.get(dom, float("nan"))
+    if stage_avg.get("score_pass2", 0.0) < 0.02 * dom_ms:
+        # the persistent kernel ran: both sweeps over K in one launch, timed in the first interval
+        dom = "score_fused_tc"
     achieved = ab["k_read"] / (dom_ms * 1e-3) / 1e9
     traffic = TRAFFIC_BYTES_PER_LAUNCH.get(dom)
     if traffic is not None:
@@ -234,8 +237,8 @@ def run_ours(args):
 
 # DRAM bytes (read + write) per launch from the ncu capture summarised under profiles/,
 # taken on a smaller case and scaled by (layers x tokens); None until captured.
-TRAFFIC_BYTES_PER_LAUNCH = {}
-TRAFFIC_CAPTURE_TOKEN_LAYERS = 1
+TRAFFIC_BYTES_PER_LAUNCH = {"score_fused_tc": 549384704}     # profiles/score_fused_tc_headline128k_2layers.txt
+TRAFFIC_CAPTURE_TOKEN_LAYERS = 2 * 131072
 
 
 def run_e2e(B, cfg, batch, p, ws, out, budget, args):

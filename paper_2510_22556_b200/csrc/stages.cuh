@@ -635,9 +635,13 @@ index_kernel(Geo g, const unsigned* __restrict__ keep_all, int keep_words, int* 
         }
     }
     for (int i = tid; i < g.window; i += kIdxThreads) oi[g.B + i] = T + i;
+    // |T*| = B (Eq. 13) whenever the scores are finite.  If the search retained fewer (scores
+    // that do not order, e.g. NaN), the rest of the list still gets valid positions, so that the
+    // gather that follows stays inside the cache, and the status word reports it.
+    for (int i = total + tid; i < g.B; i += kIdxThreads) oi[i] = 0;
     if (tid == 0) {
         out_n_keep[p] = g.B + g.window;
-        if (total != g.B) atomicOr(status, kStatInternal);      // |T*| = B (Eq. 13)
+        if (total != g.B) atomicOr(status, kStatInternal);
     }
 }
 
@@ -674,7 +678,9 @@ compact_kernel(Geo g, CompactArgs c, const int* __restrict__ out_idx, const int*
         if (r >= n_keep) break;
         const int vi = i % vec_per_row;
         const int h = vi / vec_per_head, x = vi % vec_per_head;
-        const long long tok = (long long)g.cu[seq] + oi[r];
+        const int pos = oi[r];
+        if ((unsigned)pos >= (unsigned)geo_L(g, seq)) continue;     // not a position of this sequence: row left as is
+        const long long tok = (long long)g.cu[seq] + pos;
         const uint4 val = __ldg(reinterpret_cast<const uint4*>(src + tok * s_tok + (long long)h * s_head) + x);
         reinterpret_cast<uint4*>(dst + ((size_t)p * g.n_out + r) * out_row_bytes)[vi] = val;
     }
