@@ -120,6 +120,31 @@ sablock_status_t sablock_segment(const sablock_params_t *p, const int *token_ids
                                  int *seg_id, int *seg_start, int *n_seg,
                                  void *ws, size_t ws_bytes, sablock_stream_t stream);
 
+/* Stage 1 again, for callers that have no device memory to spare for scratch and no way to get
+ * any.  (The paper has no counterpart; this is a service of this library.)  Some hosts of this
+ * code may not allocate: an inference server whose memory pool is sized once and then frozen, a
+ * plug-in that is handed only its input and output buffers, a latency-critical loop in which
+ * cudaMalloc's implicit device synchronisation is not acceptable.  This variant needs no
+ * workspace: the look-back state of the segmentation scan lives in a fixed 8.25 KB array inside the
+ * library's device image (every GPU that loads the library holds it until the process exits).
+ * Same arguments and results as sablock_segment, minus the workspace.
+ *  - Limit: T = L - W <= SABLOCK_SEGMENT_STATIC_MAX_T tokens; longer inputs are rejected with
+ *    SABLOCK_ERR_UNSUPPORTED and nothing is enqueued.
+ *  - status: dev int32[1] or NULL.  If given it must be zero before the call; a bounded wait that
+ *    ran out sets bit 0 (as in the workspace status word).  With NULL the word is kept inside the
+ *    static array and cannot be read back.
+ *  - The first call on each device looks up the array's device address (no allocation); make
+ *    that first call outside any stream capture.
+ *  - Every call on a device shares the one array.  The call clears what it needs on `stream`
+ *    before the kernel, so back-to-back calls on one stream are fine; two calls whose device work
+ *    overlaps (different streams, or different host threads on different streams) race on it and
+ *    give wrong segment ids.
+ *  - Calls no cudaMalloc / cudaFree and no allocating library routine. */
+#define SABLOCK_SEGMENT_STATIC_MAX_T (1024 * 2048)
+sablock_status_t sablock_segment_static(const sablock_params_t *p, const int *token_ids, int L,
+                                        int *seg_id, int *seg_start, int *n_seg, int *status,
+                                        sablock_stream_t stream);
+
 /* Stages 2+3 -- observation-window scoring (Sec. 3.2, Eqs. 2-4 and the per-token entropy of
  * Eq. 6) followed by segment-guided refinement (Eqs. 5-8, Algorithm 1).
  *  q_win dev [H, W, D]: queries of the last W prompt positions; k dev [L, Hkv, D];

@@ -26,7 +26,7 @@ EXPORTS = [
     "sablock_read_status", "sablock_segment", "sablock_score", "sablock_select", "sablock_compact",
     "sablock_compress", "sablock_compress_layers", "sablock_compress_layers_host", "sablock_last_launch_count",
     "sablock_params_sizeof", "sablock_workspace_region", "sablock_profile_enable", "sablock_profile_read",
-    "sablock_profile_stage_name",
+    "sablock_profile_stage_name", "sablock_segment_static",
 ]
 
 
@@ -73,6 +73,7 @@ def lib():
         l.sablock_profile_read.argtypes = [ci, vp, ci]
         l.sablock_profile_stage_name.restype = C.c_char_p
         l.sablock_segment.argtypes = [vp, vp, ci, vp, vp, vp, vp, sz, vp]
+        l.sablock_segment_static.argtypes = [vp, vp, ci, vp, vp, vp, vp, vp]
         l.sablock_score.argtypes = [vp, vp, vp, ci, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         l.sablock_select.argtypes = [vp, vp, ci, vp, vp, ci, vp, ci, vp, vp, vp, vp, sz, vp]
         l.sablock_compact.argtypes = [vp, vp, vp, ci, vp, ci, vp, vp, vp]
@@ -172,6 +173,18 @@ def segment(p: Params, token_ids: torch.Tensor, ws: torch.Tensor):
     _check(lib().sablock_segment(C.addressof(p), _ptr(token_ids), L, _ptr(seg_id), _ptr(seg_start), _ptr(n_seg),
                                  _ptr(ws), ws.numel(), _stream()), "sablock_segment")
     return seg_id, seg_start, n_seg
+
+
+SEGMENT_STATIC_MAX_T = 1024 * 2048
+
+
+def segment_static(p: Params, token_ids: torch.Tensor, seg_id: torch.Tensor, seg_start: torch.Tensor,
+                   n_seg: torch.Tensor, status: Optional[torch.Tensor] = None) -> None:
+    """sablock_segment without a workspace: the caller supplies every buffer (outputs included),
+    the scan's scratch is a fixed array inside the library.  Nothing is allocated here."""
+    _check(lib().sablock_segment_static(C.addressof(p), _ptr(token_ids), token_ids.numel(), _ptr(seg_id),
+                                        _ptr(seg_start), _ptr(n_seg), _ptr(status), _stream()),
+           "sablock_segment_static")
 
 
 def score(p: Params, q_win: torch.Tensor, k: torch.Tensor, seg_start: torch.Tensor, n_seg: torch.Tensor,

@@ -619,6 +619,54 @@ sablock_status_t sablock_segment(const sablock_params_t* p, const int* token_ids
     return run_segment(pl, p, token_ids, seg_id, seg_start, n_seg, ws, st);
 }
 
+// ---- segmentation without a workspace ---------------------------------------------------
+// Scratch of sablock_segment_static: one look-back word per 2048-token tile, then the ticket
+// counter and a private status word.  In host code this name is only a handle for the symbol
+// look-up below; the kernel gets the device address from cudaGetSymbolAddress.
+constexpr int kStaticSegTiles = SABLOCK_SEGMENT_STATIC_MAX_T / kSegTile;
+static __device__ __align__(256) unsigned long long g_segment_scratch[kStaticSegTiles + 32];
+
+sablock_status_t sablock_segment_static(const sablock_params_t* p, const int* token_ids, int L, int* seg_id,
+                                        int* seg_start, int* n_seg, int* status, sablock_stream_t stream)
+{
+    t_launches = 0;
+    if (!p || L <= p->window) return SABLOCK_ERR_INVALID_ARG;
+    SAB_TRY(validate_params(p));
+    if (!token_ids || !seg_id || !seg_start || !n_seg || !p->delim_bitmap || p->vocab_size <= 0)
+        return SABLOCK_ERR_INVALID_ARG;
+    const long long T = (long long)L - p->window;
+    if (T > SABLOCK_SEGMENT_STATIC_MAX_T) return SABLOCK_ERR_UNSUPPORTED;
+    // device address of the static array, looked up once per device with that device current
+    static unsigned long long* addr[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SABLOCK_ERR_CUDA;
+    if (!addr[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_segment_scratch) != cudaSuccess || !ptr) {
+            cudaGetLastError();
+            return SABLOCK_ERR_CUDA;
+        }
+        addr[dev] = static_cast<unsigned long long*>(ptr);
+    }
+    unsigned long long* scratch = addr[dev];
+    const int n_tiles = (int)((T + kSegTile - 1) / kSegTile);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // the array keeps the previous call's contents: tile states, ticket and private status restart at zero
+    if (cudaMemsetAsync(scratch, 0, sizeof(unsigned long long) * (size_t)n_tiles, st) != cudaSuccess ||
+        cudaMemsetAsync(scratch + kStaticSegTiles, 0, 2 * sizeof(unsigned long long), st) != cudaSuccess)
+        return SABLOCK_ERR_CUDA;
+    int* ticket = reinterpret_cast<int*>(scratch + kStaticSegTiles);
+    int* own_status = reinterpret_cast<int*>(scratch + kStaticSegTiles + 1);
+    Geo g;
+    memset(&g, 0, sizeof(g));
+    g.n_layers = g.n_seqs = 1; g.total_tokens = L; g.window = p->window;
+    g.H = p->n_q_heads; g.Hkv = p->n_kv_heads; g.D = p->head_dim; g.G = g.H / g.Hkv;
+    g.cu[0] = 0; g.cu[1] = L;
+    segment_kernel<<<dim3(n_tiles, 1), kSegThreads, 0, st>>>(g, token_ids, p->delim_bitmap, p->vocab_size, seg_id, seg_start,
+                                                             n_seg, scratch, ticket, n_tiles, status ? status : own_status);
+    return check_launch();
+}
+
 sablock_status_t sablock_score(const sablock_params_t* p, const void* q_win, const void* k, int L, const int* seg_start,
                                const int* n_seg, float* s, float* e, float* s_refined, float* seg_stats, void* ws,
                                size_t ws_bytes, sablock_stream_t stream)
