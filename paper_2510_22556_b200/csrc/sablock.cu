@@ -214,7 +214,7 @@ sablock_status_t make_plan(const sablock_params_t* p, int n_layers, int n_seqs, 
     pl->o_long_list = take(sizeof(int) * (size_t)pl->n_prob * pl->long_cap);
     pl->o_phi = take(sizeof(double) * ntok);
     pl->o_rank = take(sizeof(int) * ntok);
-    pl->o_fpart = take(pl->use_fused ? sizeof(float2) * (size_t)kFuMaxCtas * kFuPartSlots * 2 * 128 : 0);
+    pl->o_fpart = take(pl->use_fused ? sizeof(float2) * (size_t)kFuMaxCtas * kFuPartSlots * 128 : 0);
     pl->total = o;
     return SABLOCK_OK;
 }
@@ -333,7 +333,7 @@ sablock_status_t run_score(const Plan& pl, const sablock_params_t* p, const void
         const int tiles_max = (pl.max_L + kTcTile - 1) / kTcTile;
         const int min_cpp = (tiles_max + kFuMaxTilesPerCta - 1) / kFuMaxTilesPerCta;
         const int n_cta = pl.use_fused ? fused_cta_limit() : 0;
-        if (pl.use_fused && n_cta >= min_cpp) {
+        if (pl.use_fused && n_cta >= min_cpp && (long long)g.n_layers * g.total_tokens < 0x7fffffffLL) {
             int groups = n_cta / min_cpp;
             if (groups > pl.n_prob) groups = pl.n_prob;
             int cpp = n_cta / groups;

@@ -8,9 +8,8 @@
 // KV head).  A CTA owns a fixed set of token tiles of its problem and, for phase n, interleaves
 // sweep A of phase n with sweep B of phase n-1, so that the second read of a KV head's keys
 // (33.5 MB at 128K tokens) comes out of L2 shortly after the first one pulled them from HBM.
-// Between the sweeps the row sums of all CTAs of the problem are merged into log-sum-exps by
-// dedicated merge warps; CTAs hand over through two counters per phase in global memory,
-// every wait on them bounded.
+// Between the sweeps the row sums of all CTAs of the problem are merged into log-sum-exps; CTAs
+// hand over through two counters per phase in global memory, every wait on them bounded.
 //
 // Both sweeps are the same 128 x 128 x 128 product on the tensor cores with the operand roles
 // swapped: sweep A computes Q_g K^T (TMEM lane = window row, the running sum is thread-local),
@@ -19,9 +18,14 @@
 // memory (32 columns per token tile) across the KV heads of a layer, so neither the H x W x T
 // attention tensor nor \bar A ever reaches shared or global memory.
 //
-// CTA = 11 warps: warp 0 TMA producer, warp 1 MMA issuer (owns tensor memory), warps 2-9
-// epilogue (two warps per 32-lane quarter of tensor memory; in sweep A they split a tile's
-// 128 token columns, in sweep B the 32 window positions), warp 10 merges row statistics.
+// CTA = 20 warps.  Warp 0: one thread walks the work list, posts every tile step to a small ring
+// in shared memory and issues the TMA loads.  Warps 1 and 19: one MMA-issuing thread per
+// accumulator (warp 1 owns tensor memory).  Warps 2-17: epilogue, two sets of eight warps; set s
+// takes the steps whose logits land in accumulator s, so one set computes while the other waits
+// and loads.  Inside a set two warps share each 32-lane quarter of tensor memory: in sweep A they
+// split the tile's 128 token columns, in sweep B the 32 window positions.  Warp 18: hand-over
+// between CTAs (publishes this CTA's row sums, merges its share of the rows of all CTAs, fetches
+// the finished log-sum-exps), so that no epilogue thread ever waits on global memory.
 #pragma once
 #include "common.cuh"
 #include "score_simt.cuh"
@@ -29,16 +33,18 @@
 
 namespace sab {
 
-constexpr int kFuThreads = 352;
+constexpr int kFuThreads = 640;
 constexpr int kFuEpiWarp0 = 2;
-constexpr int kFuEpiThreads = 256;
-constexpr int kFuMergeWarp = 10;
+constexpr int kFuEpiWarps = 16;
+constexpr int kFuHelpWarp = 18;
+constexpr int kFuMmaWarp2 = 19;
 constexpr int kFuStages = 4;                 // K tile ring
 constexpr int kFuMaxTilesPerCta = 7;         // \bar A slots in tensor memory: 7 x 32 columns
 constexpr int kFuAbarCol0 = 256;             // columns [0, 256): two logit accumulators
 constexpr int kFuTmemCols = 512;
-constexpr int kFuLead = 3;                   // sweep A runs this many tiles ahead of sweep B
-constexpr int kFuPartSlots = 4;              // ring of per-phase partial buffers
+constexpr int kFuLead = 2;                   // sweep A runs at least this many tiles ahead of sweep B
+constexpr int kFuPartSlots = 4;              // ring of per-phase partial buffers in global memory
+constexpr int kFuLseSlots = 4;               // ring of log-sum-exp buffers in shared memory
 constexpr int kFuMaxCtasDev = 256;           // upper bound on the CTAs of one launch
 constexpr int kFuTileBytes = 2 * kAtomBytes; // 128 rows x 128 bf16
 constexpr int kFuSmemBytes = 1024 + (2 + kFuStages) * kFuTileBytes;
@@ -49,7 +55,7 @@ struct FusedArgs {
     int n_prob;
     float c2;                // log2(e) / sqrt(D)
     float eps;
-    float2* part;            // [n_groups][kFuPartSlots][cpp][2][128] row statistics (m, l)
+    float2* part;            // [n_groups][kFuPartSlots][cpp][128] row statistics (m, l)
     float* lse2;             // [n_prob][Hkv * 128] log2-sum-exp2 per window row
     int* arrive;             // [n_prob][Hkv]
     int* done;               // [n_prob][Hkv]
@@ -59,10 +65,11 @@ struct FusedArgs {
 };
 
 // Optional cycle-stamp trace of a few CTAs (compiled in with -DSABLOCK_TRACE; off otherwise):
-// role 0 = TMA producer, 1 = MMA issuer, 2 / 3 = leader thread of epilogue set 0 / 1.
+// role 0 = producer, 1 = MMA issuers (per step), 2 / 3 = first thread of epilogue set 0 / 1
+// (per own step).
 #ifdef SABLOCK_TRACE
 constexpr int kTraceOps = 600;
-__device__ long long g_trace[4][4][kTraceOps][4];   // [traced CTA][role][op][event]
+__device__ long long g_trace[4][4][kTraceOps][4];   // [traced CTA][role][step][event]
 #define FU_TRACE(role, n, ev)                                                                 \
     do {                                                                                      \
         if (tslot >= 0 && (n) < kTraceOps) g_trace[tslot][role][n][ev] = clock64();           \
@@ -78,20 +85,22 @@ struct FuBarriers {
     uint64_t tempty[2];
     uint64_t qfull[2];
     uint64_t qempty[2];
-    uint64_t sbar[2];        // the four warps of one epilogue set
+    uint64_t pbar[2][4];     // the two warps of one set that share a tensor-memory lane quarter
+    uint64_t pub_full[2];    // row sums of a phase are in shared memory (all epilogue threads)
+    uint64_t lse_full[kFuLseSlots];
     uint32_t tmem_base;
     int abort_flag;
 };
 
-// One step of a CTA's work list.
+// ---- the work list ----------------------------------------------------------------------------
 enum { kOpA = 0, kOpB = 1, kOpPairEnd = 2, kOpStop = 3 };
 
-// What a role needs to know about one phase = (problem, KV head).
+// What the producer needs to know about one phase = (problem, KV head).
 struct FuPhase {
     int phase;       // phase counter of the group; -1 = none
     int prob, j;     // problem index and KV head
-    int layer, seq;
-    int L, Tn;       // sequence length and compressible length
+    int layer;
+    int Tn;          // compressible length of the sequence
     int tok_base;    // first packed token row of the sequence
     int n_tiles;     // tiles of this CTA in the sweep in question
 };
@@ -101,12 +110,13 @@ struct FuOp {
     int k;           // which of the CTA's tiles (slot of \bar A in tensor memory)
     int tile;        // token tile index inside the sequence
     int last;        // last tile of this kind for this CTA in this phase
-    int pair;        // for kOpPairEnd: the pair that ended
+    int pair;        // the pair this step belongs to (for kOpPairEnd: the pair that ended)
 };
 
-// Deterministic walk over the work list; every role of the CTA runs its own copy.  Pair n holds
-// the sweep A tiles of phase n (`pa`) and the sweep B tiles of phase n - 1 (`pb`); all divisions
-// happen when a pair begins, the per-tile step is a few adds and compares.
+// Walk over the work list of one CTA (run by the producer thread only).  Pair n holds the sweep A
+// tiles of phase n (`pa`) and the sweep B tiles of phase n - 1 (`pb`); all divisions happen when a
+// pair begins.  Inside a pair sweep A leads by at least kFuLead tiles, and by more while the
+// log-sum-exps of phase n - 1 are not in yet (`b_ready` false).
 struct FuIter {
     const Geo& g;
     int cpp, n_groups, group, rank;
@@ -132,32 +142,34 @@ struct FuIter {
         pa.prob = group + (pair / g.Hkv) * n_groups;
         pa.j = pair % g.Hkv;
         pa.layer = pa.prob / g.n_seqs;
-        pa.seq = pa.prob % g.n_seqs;
-        pa.tok_base = g.cu[pa.seq];
-        pa.L = g.cu[pa.seq + 1] - pa.tok_base;
-        pa.Tn = pa.L - g.window;
-        if (pa.L > g.n_out) pa.n_tiles = my_tiles((pa.L + kTcTile - 1) / kTcTile);   // else: returned unchanged
+        const int seq = pa.prob % g.n_seqs;
+        pa.tok_base = g.cu[seq];
+        const int L = g.cu[seq + 1] - pa.tok_base;
+        pa.Tn = L - g.window;
+        if (L > g.n_out) pa.n_tiles = my_tiles((L + kTcTile - 1) / kTcTile);   // else: returned unchanged
     }
     __device__ void next_pair()
     {
         pb = pa;
-        pb.n_tiles = (pa.phase >= 0 && pa.L > g.n_out) ? my_tiles((pa.Tn + kTcTile - 1) / kTcTile) : 0;
+        pb.n_tiles = (pa.phase >= 0 && pa.n_tiles > 0) ? my_tiles((pa.Tn + kTcTile - 1) / kTcTile) : 0;
         ++pair; ia = ib = 0;
         load_a();
     }
-    __device__ FuOp next()
+    __device__ bool b_pending() const { return ib < pb.n_tiles; }
+    __device__ FuOp next(bool b_ready)
     {
         FuOp op;
         op.pair = pair;
         if (pair > n_phases) { op.kind = kOpStop; return op; }
-        const bool take_a = ia < pa.n_tiles && (ia < ib + kFuLead || ib >= pb.n_tiles);
+        const bool can_a = ia < pa.n_tiles, can_b = ib < pb.n_tiles;
+        const bool take_a = can_a && (!can_b || ia < ib + kFuLead || !b_ready);
         if (take_a) {
             op.kind = kOpA; op.k = ia; op.last = ia == pa.n_tiles - 1;
             op.tile = rank + ia * cpp;
             ++ia;
             return op;
         }
-        if (ib < pb.n_tiles) {
+        if (can_b) {
             op.kind = kOpB; op.k = ib; op.last = ib == pb.n_tiles - 1;
             op.tile = rank + ib * cpp;
             ++ib;
@@ -167,6 +179,30 @@ struct FuIter {
         next_pair();
         return op;
     }
+};
+
+// One tile step as the other roles see it: 16 bytes in the shared-memory ring.
+constexpr int kStepB = 1 << 0;          // sweep B (else sweep A)
+constexpr int kStepLastA = 1 << 1;      // last sweep A step of its phase for this CTA: row sums are due
+constexpr int kStepMore = 1 << 2;       // another step follows
+constexpr int kStepFirstB = 1 << 3;     // first sweep B step of its phase for this CTA: next log-sum-exp buffer
+constexpr int kStepKShift = 4;          // bits 4-6: slot of the tile among the CTA's tiles
+constexpr int kStepHead0 = 1 << 7;      // first KV head of the layer (sweep B starts \bar A afresh)
+constexpr int kStepHeadLast = 1 << 8;   // last KV head of the layer (sweep B emits s and the entropy)
+constexpr int kStepQBuf = 1 << 9;       // which query-block buffer the step's phase uses
+constexpr int kStepQPar = 1 << 10;      // parity of that buffer's load
+constexpr int kStepRel0 = 1 << 11;      // before this step: query-block buffer 0 has seen its last product
+constexpr int kStepRel1 = 1 << 12;
+constexpr int kStepMask = 1 << 13;      // sweep A tile that reaches the causal boundary
+constexpr int kStepNewQ = 1 << 14;      // first step that uses this load of the query block
+
+constexpr int kFuRing = 16;
+struct FuSched {
+    int4 ring[kFuRing];      // {flags, first token of the tile, T of the sequence, row offset of the outputs}
+    volatile int count;      // steps posted so far
+    volatile int final_;     // the producer has posted its last step
+    volatile int lse_fetched;   // log-sum-exp buffers filled so far (helper warp)
+    volatile int pub_done;      // phases whose row sums the helper warp has taken out of shared memory
 };
 
 // ---- small PTX helpers used only here -------------------------------------------------------
@@ -268,6 +304,47 @@ __device__ __forceinline__ bool wait_counter(const int* ctr, int target, volatil
     }
 }
 
+
+__device__ __forceinline__ int sched_count(const FuSched& sc)
+{
+    int v;
+    asm volatile("ld.volatile.shared.s32 %0, [%1];" : "=r"(v) : "r"(smem_u32((const void*)&sc.count)) : "memory");
+    return v;
+}
+__device__ __forceinline__ void sched_post(FuSched& sc, int idx, int4 step)
+{
+    const uint32_t dst = smem_u32(&sc.ring[idx % kFuRing]);
+    asm volatile("st.volatile.shared.v4.s32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(step.x), "r"(step.y), "r"(step.z), "r"(step.w) : "memory");
+    // shared-memory stores of one thread become visible in order: the counter after the step
+    asm volatile("st.volatile.shared.s32 [%0], %1;" ::"r"(smem_u32((const void*)&sc.count)), "r"(idx + 1) : "memory");
+}
+// Waits (bounded) until step `idx` is posted and reads it; false when there is no such step or the
+// wait gave up.
+__device__ __forceinline__ bool sched_get(FuSched& sc, int idx, int4& out, volatile int* abort_flag)
+{
+    if (sched_count(sc) <= idx) {
+        const long long t0 = clock64();
+        while (sched_count(sc) <= idx) {
+            if (sc.final_) {
+                if (sched_count(sc) <= idx) return false;
+                break;
+            }
+            if (*abort_flag || clock64() - t0 > kWaitLimitCycles) { *abort_flag = 1; return false; }
+        }
+    }
+    const uint32_t src = smem_u32(&sc.ring[idx % kFuRing]);
+    asm volatile("ld.volatile.shared.v4.s32 {%0, %1, %2, %3}, [%4];" : "=r"(out.x), "=r"(out.y), "=r"(out.z), "=r"(out.w) : "r"(src) : "memory");
+    return true;
+}
+
+// First wait of the launch that gave up: (code, CTA, warp) goes to the word after the status word.
+__device__ __forceinline__ void note_giveup(int* status, int code)
+{
+    atomicCAS(status + 1, 0, code | ((int)blockIdx.x << 8) | ((int)(threadIdx.x >> 5) << 20));
+}
+#define FU_WAIT(code, expr) ((expr) ? true : (note_giveup(fa.status, code), false))
+
+// ---- arithmetic of the epilogue ---------------------------------------------------------------
 // Sum of exp2(v * c2 - m) over 32 logits of one window row.
 __device__ __forceinline__ float chunk_expsum(const uint32_t (&r)[32], float c2, float m)
 {
@@ -306,47 +383,44 @@ struct RowSum {
     float m, l;
     bool have_m;
     __device__ void reset() { m = 0.f; l = 0.f; have_m = false; }
-    __device__ void add(const uint32_t (&r0)[32], const uint32_t (&r1)[32], float c2)
+    __device__ void add(const uint32_t (&r)[32], float c2)
     {
         if (!have_m) {
-            const float mx = fmaxf(chunk_max(r0), chunk_max(r1)) * c2;
-            m = (mx == -INFINITY) ? 0.f : ceilf(mx);
+            const float mx = chunk_max(r) * c2;
+            if (mx == -INFINITY) return;                   // nothing visible yet
+            m = ceilf(mx);
             have_m = true;
         }
-        float c = chunk_expsum(r0, c2, m) + chunk_expsum(r1, c2, m);
+        float c = chunk_expsum(r, c2, m);
         if (!(l + c < 1.8e19f)) {                          // far above the reference: move it
-            const float mx = fmaxf(chunk_max(r0), chunk_max(r1)) * c2;
-            const float m_new = fmaxf(m, ceilf(mx));
+            const float m_new = fmaxf(m, ceilf(chunk_max(r) * c2));
             l *= exp2f(m - m_new);
             m = m_new;
-            c = chunk_expsum(r0, c2, m) + chunk_expsum(r1, c2, m);
+            c = chunk_expsum(r, c2, m);
         }
         l += c;
     }
 };
 
-// accw[w] += exp2(logit * c2 - lse) for two heads' 32 window positions each (64 logits).
-__device__ __forceinline__ void accumulate_heads(float (&accw)[32], const uint32_t (&r0)[32], const uint32_t (&r1)[32],
-                                                 const float* lse0, float c2)
+// accw[i] += exp2(logit * c2 - lse) for 16 window positions of one query head.
+__device__ __forceinline__ void accumulate_head16(float (&accw)[16], const uint32_t (&r)[16], const float* lse, float c2)
 {
-    const float4* l4 = reinterpret_cast<const float4*>(lse0);
+    const float4* l4 = reinterpret_cast<const float4*>(lse);
 #pragma unroll
-    for (int i = 0; i < 32; i += 4) {
+    for (int i = 0; i < 16; i += 4) {
         const float4 ls = l4[i >> 2];
-        accw[i + 0] += ex2_approx(fmaf(__uint_as_float(r0[i + 0]), c2, -ls.x));
-        accw[i + 1] += ex2_approx(fmaf(__uint_as_float(r0[i + 1]), c2, -ls.y));
-        accw[i + 2] += ex2_approx(fmaf(__uint_as_float(r0[i + 2]), c2, -ls.z));
-        accw[i + 3] += ex2_approx(fmaf(__uint_as_float(r0[i + 3]), c2, -ls.w));
-    }
-#pragma unroll
-    for (int i = 0; i < 32; i += 4) {
-        const float4 ls = l4[8 + (i >> 2)];
-        accw[i + 0] += ex2_approx(fmaf(__uint_as_float(r1[i + 0]), c2, -ls.x));
-        accw[i + 1] += ex2_approx(fmaf(__uint_as_float(r1[i + 1]), c2, -ls.y));
-        accw[i + 2] += ex2_approx(fmaf(__uint_as_float(r1[i + 2]), c2, -ls.z));
-        accw[i + 3] += ex2_approx(fmaf(__uint_as_float(r1[i + 3]), c2, -ls.w));
+        accw[i + 0] += ex2_approx(fmaf(__uint_as_float(r[i + 0]), c2, -ls.x));
+        accw[i + 1] += ex2_approx(fmaf(__uint_as_float(r[i + 1]), c2, -ls.y));
+        accw[i + 2] += ex2_approx(fmaf(__uint_as_float(r[i + 2]), c2, -ls.z));
+        accw[i + 3] += ex2_approx(fmaf(__uint_as_float(r[i + 3]), c2, -ls.w));
     }
 }
+
+// A step as the producer holds it before posting.
+struct FuPStep {
+    int4 rec;
+    int j, layer, prob, tok_row, qseq;
+};
 
 __global__ void __launch_bounds__(kFuThreads, 1)
 score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const Geo g,
@@ -354,7 +428,10 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 {
     extern __shared__ uint8_t dyn_smem[];
     __shared__ FuBarriers sh;
-    __shared__ __align__(16) float lse_s[2][2][128];     // [epilogue set][phase parity][window row]
+    __shared__ __align__(16) FuSched sched;
+    __shared__ __align__(16) float lse_s[kFuLseSlots][128];      // log2-sum-exp2 of the window rows of a phase
+    __shared__ float2 pub_s[2][4][128];                          // [phase parity][set * 2 + half][window row]
+    __shared__ float xch[2][2][2][2][128];                       // [set][use parity][tot | ent][half][token]
     const uint32_t base = (smem_u32(dyn_smem) + 1023u) & ~1023u;
     const uint32_t q_smem = base;                                  // two query blocks
     const uint32_t k_smem = base + 2 * kFuTileBytes;               // K tile ring
@@ -367,12 +444,18 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&sh.tfull[i]), 1);
-            mbar_init(smem_u32(&sh.tempty[i]), 128);
+            mbar_init(smem_u32(&sh.tempty[i]), 256);
             mbar_init(smem_u32(&sh.qfull[i]), 1);
-            mbar_init(smem_u32(&sh.qempty[i]), 1);
-            mbar_init(smem_u32(&sh.sbar[i]), 128);
+            mbar_init(smem_u32(&sh.qempty[i]), 2);
+            mbar_init(smem_u32(&sh.pub_full[i]), kFuEpiWarps * 32);
+            for (int q = 0; q < 4; ++q) mbar_init(smem_u32(&sh.pbar[i][q]), 64);
         }
+        for (int i = 0; i < kFuLseSlots; ++i) mbar_init(smem_u32(&sh.lse_full[i]), 1);
         sh.abort_flag = 0;
+        sched.count = 0;
+        sched.final_ = 0;
+        sched.lse_fetched = 0;
+        sched.pub_done = 0;
         fence_mbar_init();
     }
     if (warp == 1) {
@@ -391,7 +474,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 #endif
 
     if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer
+        // ------------------------------------------------------------------ scheduler + TMA producer
         if (lane == 0) {
             tma_prefetch_desc(&tmQ);
             tma_prefetch_desc(&tmK);
@@ -399,257 +482,359 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             const uint64_t pol_b = l2_policy_evict_first();    // second read: last use
             const uint64_t pol_q = l2_policy_evict_last();
             FuIter it(g, fa);
-            int n_ops = 0, qloads[2] = {0, 0}, q_phase = -1;
-            while (true) {
-                const FuOp op = it.next();
-                if (op.kind == kOpStop) break;
-                if (op.kind == kOpPairEnd) continue;
-                const FuPhase& ph = op.kind == kOpA ? it.pa : it.pb;
-                if (op.kind == kOpA && ph.phase != q_phase) {      // first tile of a phase: its query block
-                    q_phase = ph.phase;
+            int q_phase = -1, vq[2] = {0, 0}, pending_rel = 0, b_idx = -1;
+            bool q_used[2] = {false, false};
+            // next step of the list with everything the other roles need folded into its flags
+            auto fetch = [&](FuPStep& e) -> bool {
+                while (true) {
+                    const bool b_ready = sched.lse_fetched > b_idx;
+                    const FuOp op = it.next(b_ready);
+                    if (op.kind == kOpStop) return false;
+                    if (op.kind == kOpPairEnd) {
+                        // the query block of phase (pair - 1) has seen its last product
+                        const int b = (op.pair - 1) & 1;
+                        if (op.pair >= 1 && q_used[b]) {
+                            pending_rel |= b ? kStepRel1 : kStepRel0;
+                            q_used[b] = false;
+                        }
+                        if (it.pb.n_tiles > 0) ++b_idx;        // the new pair's sweep B phase needs the next fetch
+                        continue;
+                    }
+                    const FuPhase& ph = op.kind == kOpA ? it.pa : it.pb;
                     const int b = ph.phase & 1;
-                    if (qloads[b] > 0 && !mbar_wait(smem_u32(&sh.qempty[b]), (qloads[b] - 1) & 1, abort_flag)) break;
-                    ++qloads[b];
+                    int flags = pending_rel | (op.k << kStepKShift) | (b ? kStepQBuf : 0);
+                    pending_rel = 0;
+                    e.qseq = -1;
+                    if (op.kind == kOpA) {
+                        if (op.last) flags |= kStepLastA;
+                        if (op.tile * kTcTile + kTcTile - 1 > ph.Tn) flags |= kStepMask;
+                        if (ph.phase != q_phase) {             // first tile of a phase: its query block
+                            q_phase = ph.phase;
+                            e.qseq = vq[b]++;
+                            q_used[b] = true;
+                            flags |= kStepNewQ;
+                        }
+                    } else {
+                        flags |= kStepB;
+                        if (op.k == 0) flags |= kStepFirstB;
+                        if (ph.j == 0) flags |= kStepHead0;
+                        if (ph.j == g.Hkv - 1) flags |= kStepHeadLast;
+                    }
+                    if ((vq[b] - 1) & 1) flags |= kStepQPar;
+                    e.rec = make_int4(flags, op.tile * kTcTile, ph.Tn, ph.layer * g.total_tokens + ph.tok_base);
+                    e.j = ph.j; e.layer = ph.layer; e.prob = ph.prob; e.tok_row = ph.tok_base + op.tile * kTcTile;
+                    return true;
+                }
+            };
+            FuPStep cur, nxt;
+            bool have = fetch(cur);
+            int n_steps = 0;
+            while (have) {
+                const bool more = fetch(nxt);
+                if (more) cur.rec.x |= kStepMore;
+                sched_post(sched, n_steps, cur.rec);
+                const bool is_b = (cur.rec.x & kStepB) != 0;
+                if (cur.qseq >= 0) {
+                    const int b = (cur.rec.x & kStepQBuf) ? 1 : 0;
+                    if (cur.qseq > 0 && !FU_WAIT(1, mbar_wait(smem_u32(&sh.qempty[b]), (cur.qseq - 1) & 1, abort_flag))) break;
                     mbar_expect_tx(smem_u32(&sh.qfull[b]), kFuTileBytes);
                     for (int a = 0; a < 2; ++a)
                         tma_load_2d(q_smem + b * kFuTileBytes + a * kAtomBytes, &tmQ, smem_u32(&sh.qfull[b]), a * 64,
-                                    ph.prob * g.H * g.window + ph.j * R, pol_q);
+                                    cur.prob * g.H * g.window + cur.j * R, pol_q);
                 }
-                const int st = n_ops % kFuStages, par = (n_ops / kFuStages) & 1;
-                FU_TRACE(0, n_ops, 0);
-                if (!mbar_wait(smem_u32(&sh.empty[st]), par ^ 1, abort_flag)) break;
-                FU_TRACE(0, n_ops, 1);
+                const int st = n_steps % kFuStages, par = (n_steps / kFuStages) & 1;
+                FU_TRACE(0, n_steps, 0);
+                if (!FU_WAIT(2, mbar_wait(smem_u32(&sh.empty[st]), par ^ 1, abort_flag))) break;
+                FU_TRACE(0, n_steps, 1);
                 mbar_expect_tx(smem_u32(&sh.full[st]), kFuTileBytes);
                 for (int a = 0; a < 2; ++a)
-                    tma_load_4d(k_smem + st * kFuTileBytes + a * kAtomBytes, &tmK, smem_u32(&sh.full[st]), a * 64, ph.j,
-                                ph.tok_base + op.tile * kTcTile, ph.layer, op.kind == kOpA ? pol_a : pol_b);
-                ++n_ops;
+                    tma_load_4d(k_smem + st * kFuTileBytes + a * kAtomBytes, &tmK, smem_u32(&sh.full[st]), a * 64, cur.j,
+                                cur.tok_row, cur.layer, is_b ? pol_b : pol_a);
+                ++n_steps;
+                cur = nxt;
+                have = more;
             }
+            sched.final_ = 1;
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
+    } else if (warp == 1 || warp == kFuMmaWarp2) {
+        // ------------------------------------------------------------------ MMA issuers
+        // One thread per accumulator: each issues the products of every other step, so that one can
+        // wait for its barriers and read its next step while the other's products run.
         if (lane == 0) {
-            FuIter it(g, fa);
-            int n_ops = 0, qwaits[2] = {0, 0}, q_phase = -1;
-            bool q_used[2] = {false, false};     // does the phase of that parity hold a query block
-            while (true) {
-                const FuOp op = it.next();
-                if (op.kind == kOpStop) break;
-                if (op.kind == kOpPairEnd) {
-                    // the query block of phase (pair - 1) has seen its last product
-                    const int b = (op.pair - 1) & 1;
-                    if (op.pair >= 1 && q_used[b]) {
-                        tc_commit(smem_u32(&sh.qempty[b]));
-                        q_used[b] = false;
+            const int acc = warp == 1 ? 0 : 1;
+            int n = 0, n_mine = 0, q_gen[2] = {0, 0}, q_seen[2] = {0, 0};
+            int4 e;
+            while (sched_get(sched, n, e, abort_flag)) {
+                const int flags = e.x;
+                if (flags & kStepRel0) tc_commit(smem_u32(&sh.qempty[0]));
+                if (flags & kStepRel1) tc_commit(smem_u32(&sh.qempty[1]));
+                const int b = (flags & kStepQBuf) ? 1 : 0;
+                if (flags & kStepNewQ) ++q_gen[b];
+                const bool mine = (n & 1) == acc;
+                const int st = n % kFuStages, par = (n / kFuStages) & 1;
+                if (mine) {
+                    FU_TRACE(1, n, 0);
+                    if (q_seen[b] != q_gen[b]) {                   // this load of the query block
+                        q_seen[b] = q_gen[b];
+                        if (!FU_WAIT(3, mbar_wait(smem_u32(&sh.qfull[b]), (flags & kStepQPar) ? 1u : 0u, abort_flag))) break;
                     }
-                    continue;
+                    if (!FU_WAIT(4, mbar_wait(smem_u32(&sh.tempty[acc]), (uint32_t)((n_mine & 1) ^ 1), abort_flag))) break;
+                    if (!FU_WAIT(5, mbar_wait(smem_u32(&sh.full[st]), (uint32_t)par, abort_flag))) break;
+                    FU_TRACE(1, n, 1);
+                    tc_fence_after();
+                    const uint32_t kt = k_smem + st * kFuTileBytes, qt = q_smem + b * kFuTileBytes;
+                    if (flags & kStepB) tc_issue_tile(tmem, acc, kt, qt, 8);      // rows = tokens
+                    else                tc_issue_tile(tmem, acc, qt, kt, 8);      // rows = window rows
+                    FU_TRACE(1, n, 2);
+                    tc_commit(smem_u32(&sh.empty[st]));
+                    tc_commit(smem_u32(&sh.tfull[acc]));
+                    FU_TRACE(1, n, 3);
+                    ++n_mine;
                 }
-                const FuPhase& ph = op.kind == kOpA ? it.pa : it.pb;
-                const int b = ph.phase & 1;
-                if (op.kind == kOpA && ph.phase != q_phase) {
-                    q_phase = ph.phase;
-                    if (!mbar_wait(smem_u32(&sh.qfull[b]), qwaits[b] & 1, abort_flag)) break;
-                    ++qwaits[b];
-                    q_used[b] = true;
-                }
-                const int st = n_ops % kFuStages, par = (n_ops / kFuStages) & 1;
-                const int acc = n_ops & 1, aph = (n_ops >> 1) & 1;
-                FU_TRACE(1, n_ops, 0);
-                if (!mbar_wait(smem_u32(&sh.tempty[acc]), aph ^ 1, abort_flag)) break;
-                FU_TRACE(1, n_ops, 1);
-                if (!mbar_wait(smem_u32(&sh.full[st]), par, abort_flag)) break;
-                FU_TRACE(1, n_ops, 2);
-                tc_fence_after();
-                const uint32_t kt = k_smem + st * kFuTileBytes, qt = q_smem + b * kFuTileBytes;
-                if (op.kind == kOpA) tc_issue_tile(tmem, acc, qt, kt, 8);     // rows = window rows
-                else                 tc_issue_tile(tmem, acc, kt, qt, 8);     // rows = tokens
-                tc_commit(smem_u32(&sh.empty[st]));
-                tc_commit(smem_u32(&sh.tfull[acc]));
-                ++n_ops;
+                ++n;
+                if (!(flags & kStepMore)) break;
             }
         }
-    } else if (warp == kFuMergeWarp) {
-        // ------------------------------------------------------------------ row-statistics merge
-        FuIter it(g, fa);
-        const int group = it.group, rank = it.rank;
-        for (int phase = 0; phase < it.n_phases; ++phase) {
+    } else if (warp == kFuHelpWarp) {
+        // ------------------------------------------------------------------ hand-over between CTAs
+        // Per phase, in this order: publish this CTA's row sums (the epilogue left the four (set, half)
+        // partial sums of every window row in shared memory), merge the sums of all CTAs for this
+        // CTA's share of the rows, fetch the finished log-sum-exps for this CTA's sweep B.
+        const int group = blockIdx.x / fa.cpp, rank = blockIdx.x % fa.cpp;
+        const int my_probs = group < fa.n_groups ? (fa.n_prob - group + fa.n_groups - 1) / fa.n_groups : 0;
+        const int n_phases = my_probs * g.Hkv;
+        const int n_mergers = min(fa.cpp, R);
+        int n_fetch = 0, n_pub = 0;
+        for (int phase = 0; phase < n_phases; ++phase) {
             const int prob = group + (phase / g.Hkv) * fa.n_groups, j = phase % g.Hkv, seq = prob % g.n_seqs;
             if (geo_identity(g, seq)) continue;
-            const int nt1 = (geo_L(g, seq) + kTcTile - 1) / kTcTile;
-            const int n_src = 2 * min(fa.cpp, nt1);             // (CTA that holds tiles, epilogue set)
-            if (rank >= R) continue;
+            const int L = geo_L(g, seq);
+            const int nt1 = (L + kTcTile - 1) / kTcTile, nt2 = (L - g.window + kTcTile - 1) / kTcTile;
+            const int n_src = min(fa.cpp, nt1);                 // CTAs that hold tiles of this problem
             bool ok = true;
-            if (lane == 0) ok = wait_counter(fa.arrive + prob * g.Hkv + j, n_src, abort_flag, fa.status);
-            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-            if (!ok) break;
-            const float2* pp = fa.part + ((size_t)group * kFuPartSlots + (phase % kFuPartSlots)) * fa.cpp * 2 * R;
-            for (int row = rank; row < R; row += fa.cpp) {
-                // partial i = (source CTA, epilogue set), merged in index order; all loads of a
-                // lane are issued before the first use so that their latencies overlap
-                constexpr int kPer = 2 * kFuMaxCtasDev / 32;
-                float2 v[kPer];
-#pragma unroll
-                for (int u = 0; u < kPer; ++u) {
-                    const int i = lane + 32 * u;
-                    v[u] = i < n_src ? __ldcg(pp + (size_t)i * R + row) : make_float2(0.f, 0.f);
+            if (rank < nt1) {
+                // the slot of the partial ring is free once the phase that used it last is merged
+                if (lane == 0 && phase >= kFuPartSlots) {
+                    const int old = phase - kFuPartSlots;
+                    ok = FU_WAIT(11, wait_counter(fa.done + (group + (old / g.Hkv) * fa.n_groups) * g.Hkv + old % g.Hkv, n_mergers,
+                                                  abort_flag, fa.status));
                 }
-                float m = -INFINITY;
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                if (!ok) break;
+                const int buf = n_pub & 1;
+                if (!FU_WAIT(6, mbar_wait(smem_u32(&sh.pub_full[buf]), (uint32_t)((n_pub >> 1) & 1), abort_flag))) break;
+                float2* dst = fa.part + (((size_t)group * kFuPartSlots + (phase % kFuPartSlots)) * fa.cpp + rank) * R;
 #pragma unroll
-                for (int u = 0; u < kPer; ++u)
-                    if (v[u].y > 0.f) m = fmaxf(m, v[u].x);
+                for (int u = 0; u < 4; ++u) {
+                    const int row = lane + 32 * u;
+                    float m = -INFINITY;
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-                float l = 0.f;
+                    for (int x = 0; x < 4; ++x) {
+                        const float2 v = pub_s[buf][x][row];
+                        if (v.y > 0.f) m = fmaxf(m, v.x);
+                    }
+                    float l = 0.f;
 #pragma unroll
-                for (int u = 0; u < kPer; ++u)
-                    if (v[u].y > 0.f) l += v[u].y * exp2f(v[u].x - m);
-                l = warp_sum(l);
-                if (lane == 0) fa.lse2[(size_t)prob * g.H * g.window + j * R + row] = m + log2f(l);
-            }
-            __syncwarp();
-            if (lane == 0) {
+                    for (int x = 0; x < 4; ++x) {
+                        const float2 v = pub_s[buf][x][row];
+                        if (v.y > 0.f) l += v.y * exp2f(v.x - m);     // exponents are integers: exact scaling
+                    }
+                    dst[row] = make_float2(l > 0.f ? m : 0.f, l);
+                }
                 __threadfence();
-                atomicAdd(fa.done + prob * g.Hkv + j, 1);
+                __syncwarp();
+                ++n_pub;
+                if (lane == 0) {
+                    sched.pub_done = n_pub;
+                    atomicAdd(fa.arrive + prob * g.Hkv + j, 1);
+                }
+            }
+            if (rank < R) {
+                if (lane == 0) ok = FU_WAIT(12, wait_counter(fa.arrive + prob * g.Hkv + j, n_src, abort_flag, fa.status));
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                if (!ok) break;
+                const float2* pp = fa.part + ((size_t)group * kFuPartSlots + (phase % kFuPartSlots)) * fa.cpp * R;
+                for (int row = rank; row < R; row += fa.cpp) {
+                    // one partial per source CTA, merged in index order; all loads of a lane are issued
+                    // before the first use so that their latencies overlap
+                    constexpr int kPer = kFuMaxCtasDev / 32;
+                    float2 v[kPer];
+#pragma unroll
+                    for (int u = 0; u < kPer; ++u) {
+                        const int i = lane + 32 * u;
+                        v[u] = i < n_src ? __ldcg(pp + (size_t)i * R + row) : make_float2(0.f, 0.f);
+                    }
+                    float m = -INFINITY;
+#pragma unroll
+                    for (int u = 0; u < kPer; ++u)
+                        if (v[u].y > 0.f) m = fmaxf(m, v[u].x);
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+                    float l = 0.f;
+#pragma unroll
+                    for (int u = 0; u < kPer; ++u)
+                        if (v[u].y > 0.f) l += v[u].y * exp2f(v[u].x - m);
+                    l = warp_sum(l);
+                    if (lane == 0) fa.lse2[(size_t)prob * g.H * g.window + j * R + row] = m + log2f(l);
+                }
+                __syncwarp();
+                if (lane == 0) {
+                    __threadfence();
+                    atomicAdd(fa.done + prob * g.Hkv + j, 1);
+                }
+            }
+            // the finished log-sum-exps, if this CTA runs sweep B for the phase
+            if (rank < nt2) {
+                if (lane == 0) ok = FU_WAIT(13, wait_counter(fa.done + prob * g.Hkv + j, n_mergers, abort_flag, fa.status));
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                if (!ok) break;
+                const int slot = n_fetch % kFuLseSlots;
+                const float* src = fa.lse2 + (size_t)prob * g.H * g.window + j * R;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) lse_s[slot][lane + 32 * u] = __ldcg(src + lane + 32 * u);
+                __syncwarp();
+                ++n_fetch;
+                if (lane == 0) {
+                    mbar_arrive(smem_u32(&sh.lse_full[slot]));
+                    sched.lse_fetched = n_fetch;
+                }
             }
         }
-    } else if (warp >= kFuEpiWarp0 && warp < kFuEpiWarp0 + 8) {
+    } else if (warp >= kFuEpiWarp0 && warp < kFuEpiWarp0 + kFuEpiWarps) {
         // ------------------------------------------------------------------ epilogue
-        // Two sets of four warps; set s takes the tiles whose logits land in accumulator s, so
-        // the sets run half a tile out of step and one computes while the other waits and loads.
         const int ew = warp - kFuEpiWarp0;
         const int q4 = warp & 3;                       // tensor-memory lane quarter of this warp
-        const int set = ew >> 2;
+        const int set = (ew >> 2) & 1;
+        const int half = ew >> 3;
         const int row = q4 * 32 + lane;                // TMEM lane: window row (sweep A) or token (sweep B)
-        const bool leader = (ew & 3) == 0 && lane == 0;
+        const bool first_thread = (ew & 11) == 0 && lane == 0;       // for the trace
+        (void)first_thread;
         const uint32_t lane_addr = tmem + ((uint32_t)(q4 * 32) << 16);
         const uint32_t acc_addr = lane_addr + (uint32_t)set * 128u;
         const float c2 = fa.c2;
         const float inv_H = 1.f / (float)g.H;
-        const int n_mergers = min(fa.cpp, R);
-        FuIter it(g, fa);
-        const int group = it.group, rank = it.rank;
-        RowSum rs;                                     // sweep A state of this window row in this set
+        RowSum rs;                                     // sweep A state of (window row, set, half)
         rs.reset();
-        int n_ops = 0, n_mine = 0, lse_phase = -1, n_sync = 0;
-        while (true) {
-            const FuOp op = it.next();
-            if (op.kind == kOpStop) break;
-            if (op.kind == kOpPairEnd) continue;
-            const bool mine = (n_ops & 1) == set;
-            ++n_ops;
-            if (op.kind == kOpA) {
-                const FuPhase& ph = it.pa;
+        int n = 0, n_mine = 0, n_lse = -1, lse_waited = -1, n_pub = 0, n_psync = 0, n_fin = 0;
+        int4 e;
+        while (sched_get(sched, n, e, abort_flag)) {
+            const int flags = e.x;
+            const bool mine = (n & 1) == set;
+            ++n;
+            if (!(flags & kStepB)) {
                 if (mine) {
-                    if (leader) FU_TRACE(2 + set, n_mine, 0);
-                    if (!mbar_wait(smem_u32(&sh.tfull[set]), n_mine & 1, abort_flag)) break;
-                    if (leader) FU_TRACE(2 + set, n_mine, 1);
+                    if (first_thread) FU_TRACE(2 + set, n_mine, 0);
+                    if (!FU_WAIT(7, mbar_wait(smem_u32(&sh.tfull[set]), (uint32_t)(n_mine & 1), abort_flag))) break;
+                    if (first_thread) FU_TRACE(2 + set, n_mine, 1);
                     tc_fence_after();
-                    const int tok0 = op.tile * kTcTile;
-                    const int lim = ph.Tn + (row & 31);            // causal: key index <= T + w (Eq. 2)
-                    const bool need_mask = tok0 + 127 > ph.Tn;
                     uint32_t r0[32], r1[32];
-                    tmem_ld32_issue(acc_addr, r0);
-                    tmem_ld32_issue(acc_addr + 32, r1);
-                    tmem_ld_wait();
-                    if (need_mask) { chunk_mask(r0, tok0, lim); chunk_mask(r1, tok0 + 32, lim); }
-                    rs.add(r0, r1, c2);
-                    tmem_ld32_issue(acc_addr + 64, r0);
-                    tmem_ld32_issue(acc_addr + 96, r1);
+                    tmem_ld32_issue(acc_addr + half * 64, r0);
+                    tmem_ld32_issue(acc_addr + half * 64 + 32, r1);
                     tmem_ld_wait();
                     tc_fence_before();
                     mbar_arrive(smem_u32(&sh.tempty[set]));        // logits are in registers: release the accumulator
-                    if (leader) FU_TRACE(2 + set, n_mine, 2);
-                    if (need_mask) { chunk_mask(r0, tok0 + 64, lim); chunk_mask(r1, tok0 + 96, lim); }
-                    rs.add(r0, r1, c2);
-                    if (leader) FU_TRACE(2 + set, n_mine, 3);
+                    if (first_thread) FU_TRACE(2 + set, n_mine, 2);
+                    if (flags & kStepMask) {
+                        const int tok0 = e.y + half * 64;
+                        const int lim = e.z + (row & 31);          // causal: key index <= T + w (Eq. 2)
+                        chunk_mask(r0, tok0, lim);
+                        chunk_mask(r1, tok0 + 32, lim);
+                    }
+                    rs.add(r0, c2);
+                    rs.add(r1, c2);
+                    if (first_thread) FU_TRACE(2 + set, n_mine, 3);
                     ++n_mine;
                 }
-                if (op.last) {
-                    // Publish this set's row sums of the phase.  The partial buffers are a ring over
-                    // phases: the slot is free once every merge of the phase that used it last is
-                    // done.  (A CTA that also runs sweep B is throttled by it anyway; one that owns
-                    // only a window tile is not.)
-                    if (leader && ph.phase >= kFuPartSlots) {
-                        const int old = ph.phase - kFuPartSlots;
-                        wait_counter(fa.done + (group + (old / g.Hkv) * fa.n_groups) * g.Hkv + old % g.Hkv, n_mergers,
-                                     abort_flag, fa.status);
+                if (flags & kStepLastA) {
+                    // Hand this thread's row sum of the phase to the helper warp (no waiting unless the
+                    // helper is two phases behind).
+                    const int buf = n_pub & 1;
+                    if (n_pub >= 2 && sched.pub_done < n_pub - 1) {
+                        const long long t0 = clock64();
+                        while (sched.pub_done < n_pub - 1) {
+                            if (*abort_flag || clock64() - t0 > kWaitLimitCycles) { note_giveup(fa.status, 21); *abort_flag = 1; break; }
+                        }
+                        if (*abort_flag) break;
                     }
-                    if (!group_sync(&sh.sbar[set], n_sync, abort_flag)) break;
-                    float2* pp = fa.part + ((size_t)group * kFuPartSlots + (ph.phase % kFuPartSlots)) * fa.cpp * 2 * R;
-                    pp[((size_t)rank * 2 + set) * R + row] = make_float2(rs.m, rs.l);
-                    __threadfence();
-                    if (!group_sync(&sh.sbar[set], n_sync, abort_flag)) break;
-                    if (leader) atomicAdd(fa.arrive + ph.prob * g.Hkv + ph.j, 1);
+                    pub_s[buf][set * 2 + half][row] = make_float2(rs.m, rs.l);
+                    mbar_arrive(smem_u32(&sh.pub_full[buf]));
+                    ++n_pub;
                     rs.reset();
                 }
-            } else if (mine) {
-                const FuPhase& ph = it.pb;
-                if (ph.phase != lse_phase) {                       // log-sum-exps of this phase
-                    lse_phase = ph.phase;
-                    if (leader) wait_counter(fa.done + ph.prob * g.Hkv + ph.j, n_mergers, abort_flag, fa.status);
-                    if (!group_sync(&sh.sbar[set], n_sync, abort_flag)) break;
-                    lse_s[set][ph.phase & 1][row] = __ldcg(fa.lse2 + (size_t)ph.prob * g.H * g.window + ph.j * R + row);
-                    if (!group_sync(&sh.sbar[set], n_sync, abort_flag)) break;
-                }
-                if (leader) FU_TRACE(2 + set, n_mine, 0);
-                if (!mbar_wait(smem_u32(&sh.tfull[set]), n_mine & 1, abort_flag)) break;
-                if (leader) FU_TRACE(2 + set, n_mine, 1);
-                tc_fence_after();
-                const float* lj = lse_s[set][ph.phase & 1];
-                float accw[32];
+            } else {
+                if (flags & kStepFirstB) ++n_lse;                  // n_lse-th phase in which this CTA runs sweep B
+                if (mine) {
+                    if (n_lse != lse_waited) {                     // log-sum-exps of this phase (fetched by warp 18)
+                        lse_waited = n_lse;
+                        if (!FU_WAIT(8, mbar_wait(smem_u32(&sh.lse_full[n_lse % kFuLseSlots]), (uint32_t)((n_lse / kFuLseSlots) & 1), abort_flag)))
+                            break;
+                    }
+                    if (first_thread) FU_TRACE(2 + set, n_mine, 0);
+                    if (!FU_WAIT(7, mbar_wait(smem_u32(&sh.tfull[set]), (uint32_t)(n_mine & 1), abort_flag))) break;
+                    if (first_thread) FU_TRACE(2 + set, n_mine, 1);
+                    tc_fence_after();
+                    const float* lj = lse_s[n_lse % kFuLseSlots] + half * 16;
+                    float accw[16];
 #pragma unroll
-                for (int i = 0; i < 32; ++i) accw[i] = 0.f;
-                uint32_t r0[32], r1[32];
-                tmem_ld32_issue(acc_addr, r0);                     // query heads 0, 1 of the group
-                tmem_ld32_issue(acc_addr + 32, r1);
-                tmem_ld_wait();
-                accumulate_heads(accw, r0, r1, lj, c2);
-                tmem_ld32_issue(acc_addr + 64, r0);                // query heads 2, 3
-                tmem_ld32_issue(acc_addr + 96, r1);
-                tmem_ld_wait();
-                tc_fence_before();
-                mbar_arrive(smem_u32(&sh.tempty[set]));
-                if (leader) FU_TRACE(2 + set, n_mine, 2);
-                accumulate_heads(accw, r0, r1, lj + 64, c2);
-                const int n_this = n_mine;
-                ++n_mine;
-                // \bar A of this token tile, summed over the KV heads seen so far
-                const uint32_t abar_addr = lane_addr + (uint32_t)(kFuAbarCol0 + op.k * 32);
-                if (ph.j > 0) {
-                    tmem_ld32_issue(abar_addr, r0);
+                    for (int i = 0; i < 16; ++i) accw[i] = 0.f;
+                    uint32_t v0[16], v1[16], v2[16], v3[16];       // query head hl of the group, 16 window positions
+                    tmem_ld16_issue(acc_addr + half * 16, v0);
+                    tmem_ld16_issue(acc_addr + 32 + half * 16, v1);
+                    tmem_ld16_issue(acc_addr + 64 + half * 16, v2);
+                    tmem_ld16_issue(acc_addr + 96 + half * 16, v3);
                     tmem_ld_wait();
+                    tc_fence_before();
+                    mbar_arrive(smem_u32(&sh.tempty[set]));
+                    if (first_thread) FU_TRACE(2 + set, n_mine, 2);
+                    accumulate_head16(accw, v0, lj, c2);
+                    accumulate_head16(accw, v1, lj + 32, c2);
+                    accumulate_head16(accw, v2, lj + 64, c2);
+                    accumulate_head16(accw, v3, lj + 96, c2);
+                    // \bar A of this token tile, summed over the KV heads seen so far
+                    const uint32_t abar_addr = lane_addr + (uint32_t)(kFuAbarCol0 + ((flags >> kStepKShift) & 7) * 32 + half * 16);
+                    if (!(flags & kStepHead0)) {
+                        tmem_ld16_issue(abar_addr, v0);
+                        tmem_ld_wait();
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) accw[i] += __uint_as_float(r0[i]);
-                }
-                if (ph.j < g.Hkv - 1) {
-                    tmem_st32(abar_addr, accw);
-                    tmem_st_wait();
-                    tc_fence_before();         // the next head's update may come from the other set's warps
-                } else {
-                    // last KV head of the layer: s_t (Eqs. 3, 4) and the entropy of Eq. 6
-                    float t0 = 0.f, t1 = 0.f, t2 = 0.f, t3 = 0.f;
+                        for (int i = 0; i < 16; ++i) accw[i] += __uint_as_float(v0[i]);
+                    }
+                    if (!(flags & kStepHeadLast)) {
+                        tmem_st16(abar_addr, accw);
+                        tmem_st_wait();
+                        tc_fence_before();         // the next head's update may come from the other set's warps
+                    } else {
+                        // last KV head of the layer: s_t (Eqs. 3, 4) and the entropy of Eq. 6; the two warps
+                        // that hold the halves of a token's window positions exchange partial sums
+                        const int par = n_fin & 1;
+                        ++n_fin;
+                        float t0 = 0.f, t1 = 0.f;
 #pragma unroll
-                    for (int i = 0; i < 32; i += 4) { t0 += accw[i]; t1 += accw[i + 1]; t2 += accw[i + 2]; t3 += accw[i + 3]; }
-                    const float tot = (t0 + t1) + (t2 + t3);
-                    float ent = 0.f;
-                    if (tot > 0.f) {
-                        const float inv = 1.f / tot;
+                        for (int i = 0; i < 16; i += 2) { t0 += accw[i]; t1 += accw[i + 1]; }
+                        xch[set][par][0][half][row] = t0 + t1;
+                        if (!FU_WAIT(20, group_sync(&sh.pbar[set][q4], n_psync, abort_flag))) break;
+                        const float tot = xch[set][par][0][0][row] + xch[set][par][0][1][row];
+                        float ent_h = 0.f;
+                        if (tot > 0.f) {
+                            const float inv = 1.f / tot;
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) {
-                            const float ah = accw[i] * inv;                       // \hat A (Eq. 6)
-                            ent -= ah * (lg2_approx(ah + fa.eps) * 0.6931471805599453f);
+                            for (int i = 0; i < 16; ++i) {
+                                const float ah = accw[i] * inv;                       // \hat A (Eq. 6)
+                                ent_h -= ah * (lg2_approx(ah + fa.eps) * 0.6931471805599453f);
+                            }
+                        }
+                        xch[set][par][1][half][row] = ent_h;
+                        if (!FU_WAIT(20, group_sync(&sh.pbar[set][q4], n_psync, abort_flag))) break;
+                        const int t = e.y + row;
+                        if (half == 0 && t < e.z) {
+                            fa.s_out[(size_t)e.w + t] = tot * inv_H;
+                            fa.e_out[(size_t)e.w + t] = xch[set][par][1][0][row] + xch[set][par][1][1][row];
                         }
                     }
-                    const int t = op.tile * kTcTile + row;
-                    if (t < ph.Tn) {
-                        const size_t off = (size_t)ph.layer * g.total_tokens + ph.tok_base;
-                        fa.s_out[off + t] = tot * inv_H;
-                        fa.e_out[off + t] = ent;
-                    }
+                    if (first_thread) FU_TRACE(2 + set, n_mine, 3);
+                    ++n_mine;
                 }
-                if (leader) FU_TRACE(2 + set, n_this, 3);
-                (void)n_this;
             }
+            if (!(flags & kStepMore)) break;
         }
     }
 
