@@ -38,7 +38,8 @@ constexpr int kFuEpiWarp0 = 2;
 constexpr int kFuEpiWarps = 16;
 constexpr int kFuHelpWarp = 18;
 constexpr int kFuMmaWarp2 = 19;
-constexpr int kFuStages = 4;                 // K tile ring
+constexpr int kFuStages = 3;                 // K tile ring
+constexpr int kFuQBufs = 3;                  // query-block buffers: phases n - 1 (sweep B), n (sweep A), n + 1 (loading ahead)
 constexpr int kFuMaxTilesPerCta = 7;         // \bar A slots in tensor memory: 7 x 32 columns
 constexpr int kFuAbarCol0 = 256;             // columns [0, 256): two logit accumulators
 constexpr int kFuTmemCols = 512;
@@ -47,7 +48,16 @@ constexpr int kFuPartSlots = 4;              // ring of per-phase partial buffer
 constexpr int kFuLseSlots = 4;               // ring of log-sum-exp buffers in shared memory
 constexpr int kFuMaxCtasDev = 256;           // upper bound on the CTAs of one launch
 constexpr int kFuTileBytes = 2 * kAtomBytes; // 128 rows x 128 bf16
-constexpr int kFuSmemBytes = 1024 + (2 + kFuStages) * kFuTileBytes;
+constexpr int kFuSmemBytes = 1024 + (kFuQBufs + kFuStages) * kFuTileBytes;
+#ifndef SABLOCK_RELEASE_AT
+#define SABLOCK_RELEASE_AT 0
+#endif
+// When an epilogue set hands its accumulator back to the MMA issuer: 0 = as soon as the logits
+// are in registers, 1 = after half of the step's arithmetic, 2 = when the step is done.  A late
+// release makes the tensor core pace the sets: their products cannot overlap, so the two sets
+// settle half a step apart and one computes while the other waits, loads and fetches its next
+// step, instead of both doing so at the same time.
+constexpr int kReleaseAt = SABLOCK_RELEASE_AT;
 
 struct FusedArgs {
     int cpp;                 // CTAs per group (one group works on one problem at a time)
@@ -83,8 +93,8 @@ struct FuBarriers {
     uint64_t empty[kFuStages];
     uint64_t tfull[2];
     uint64_t tempty[2];
-    uint64_t qfull[2];
-    uint64_t qempty[2];
+    uint64_t qfull[kFuQBufs];
+    uint64_t qempty[kFuQBufs];
     uint64_t pbar[2][4];     // the two warps of one set that share a tensor-memory lane quarter
     uint64_t pub_full[2];    // row sums of a phase are in shared memory (all epilogue threads)
     uint64_t lse_full[kFuLseSlots];
@@ -122,6 +132,7 @@ struct FuIter {
     int cpp, n_groups, group, rank;
     int n_phases;            // phases of this group
     int pair, ia, ib;
+    int tiles_b;             // sweep B tiles of this CTA in pa's problem
     FuPhase pa, pb;
     __device__ FuIter(const Geo& geo, const FusedArgs& a) : g(geo), cpp(a.cpp), n_groups(a.n_groups)
     {
@@ -129,29 +140,33 @@ struct FuIter {
         rank = blockIdx.x % cpp;
         const int my_probs = group < n_groups ? (a.n_prob - group + n_groups - 1) / n_groups : 0;
         n_phases = my_probs * g.Hkv;
-        pair = 0; ia = ib = 0;
+        pair = 0; ia = ib = 0; tiles_b = 0;
         pb.phase = -1; pb.n_tiles = 0;
+        pa.j = 0; pa.prob = group; pa.n_tiles = 0;
         load_a();
     }
     __device__ int my_tiles(int n) const { return rank < n ? (n - rank + cpp - 1) / cpp : 0; }
+    // Phase `pair` for sweep A.  Consecutive phases of a problem differ only in the KV head; the
+    // divisions are paid once per problem.
     __device__ void load_a()
     {
         pa.phase = pair;
-        pa.n_tiles = 0;
-        if (pair >= n_phases) { pa.phase = -1; return; }
-        pa.prob = group + (pair / g.Hkv) * n_groups;
-        pa.j = pair % g.Hkv;
+        if (pair >= n_phases) { pa.phase = -1; pa.n_tiles = 0; return; }
+        if (pair > 0 && pa.j + 1 < g.Hkv) { ++pa.j; return; }           // same problem, next KV head
+        pa.prob = pair == 0 ? group : pa.prob + n_groups;
+        pa.j = 0;
         pa.layer = pa.prob / g.n_seqs;
-        const int seq = pa.prob % g.n_seqs;
+        const int seq = pa.prob - pa.layer * g.n_seqs;
         pa.tok_base = g.cu[seq];
         const int L = g.cu[seq + 1] - pa.tok_base;
         pa.Tn = L - g.window;
-        if (L > g.n_out) pa.n_tiles = my_tiles((L + kTcTile - 1) / kTcTile);   // else: returned unchanged
+        pa.n_tiles = L > g.n_out ? my_tiles((L + kTcTile - 1) / kTcTile) : 0;   // else: returned unchanged
+        tiles_b = pa.n_tiles > 0 ? my_tiles((pa.Tn + kTcTile - 1) / kTcTile) : 0;
     }
     __device__ void next_pair()
     {
         pb = pa;
-        pb.n_tiles = (pa.phase >= 0 && pa.n_tiles > 0) ? my_tiles((pa.Tn + kTcTile - 1) / kTcTile) : 0;
+        pb.n_tiles = pa.phase >= 0 ? tiles_b : 0;
         ++pair; ia = ib = 0;
         load_a();
     }
@@ -189,12 +204,11 @@ constexpr int kStepFirstB = 1 << 3;     // first sweep B step of its phase for t
 constexpr int kStepKShift = 4;          // bits 4-6: slot of the tile among the CTA's tiles
 constexpr int kStepHead0 = 1 << 7;      // first KV head of the layer (sweep B starts \bar A afresh)
 constexpr int kStepHeadLast = 1 << 8;   // last KV head of the layer (sweep B emits s and the entropy)
-constexpr int kStepQBuf = 1 << 9;       // which query-block buffer the step's phase uses
-constexpr int kStepQPar = 1 << 10;      // parity of that buffer's load
-constexpr int kStepRel0 = 1 << 11;      // before this step: query-block buffer 0 has seen its last product
-constexpr int kStepRel1 = 1 << 12;
-constexpr int kStepMask = 1 << 13;      // sweep A tile that reaches the causal boundary
-constexpr int kStepNewQ = 1 << 14;      // first step that uses this load of the query block
+constexpr int kStepQBufShift = 9;       // bits 9-10: which query-block buffer the step's phase uses
+constexpr int kStepQPar = 1 << 11;      // parity of that buffer's load
+constexpr int kStepRelShift = 12;       // bits 12-14: before this step, query-block buffer i has seen its last product
+constexpr int kStepMask = 1 << 15;      // sweep A tile that reaches the causal boundary
+constexpr int kStepNewQ = 1 << 16;      // first step that uses this load of the query block
 
 constexpr int kFuRing = 16;
 struct FuSched {
@@ -391,14 +405,17 @@ struct RowSum {
             m = ceilf(mx);
             have_m = true;
         }
-        float c = chunk_expsum(r, c2, m);
-        if (!(l + c < 1.8e19f)) {                          // far above the reference: move it
+        // one copy of the summation code: the loop repeats only when the sum would leave the
+        // fp32 range, after moving the reference exponent up to the chunk's maximum
+#pragma unroll 1
+        while (true) {
+            const float c = chunk_expsum(r, c2, m);
+            if (l + c < 1.8e19f || !(c == c)) { l += c; break; }
             const float m_new = fmaxf(m, ceilf(chunk_max(r) * c2));
+            if (!(m_new > m)) { l += c; break; }            // cannot be improved (non-finite logits)
             l *= exp2f(m - m_new);
             m = m_new;
-            c = chunk_expsum(r, c2, m);
         }
-        l += c;
     }
 };
 
@@ -419,7 +436,7 @@ __device__ __forceinline__ void accumulate_head16(float (&accw)[16], const uint3
 // A step as the producer holds it before posting.
 struct FuPStep {
     int4 rec;
-    int j, layer, prob, tok_row, qseq;
+    int j, layer, prob, tok_row, qseq, phase;
 };
 
 __global__ void __launch_bounds__(kFuThreads, 1)
@@ -433,8 +450,8 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     __shared__ float2 pub_s[2][4][128];                          // [phase parity][set * 2 + half][window row]
     __shared__ float xch[2][2][2][2][128];                       // [set][use parity][tot | ent][half][token]
     const uint32_t base = (smem_u32(dyn_smem) + 1023u) & ~1023u;
-    const uint32_t q_smem = base;                                  // two query blocks
-    const uint32_t k_smem = base + 2 * kFuTileBytes;               // K tile ring
+    const uint32_t q_smem = base;                                  // query blocks
+    const uint32_t k_smem = base + kFuQBufs * kFuTileBytes;        // K tile ring
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (warp == 0 && lane == 0) {
@@ -442,11 +459,13 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             mbar_init(smem_u32(&sh.full[i]), 1);
             mbar_init(smem_u32(&sh.empty[i]), 1);
         }
+        for (int i = 0; i < kFuQBufs; ++i) {
+            mbar_init(smem_u32(&sh.qfull[i]), 1);
+            mbar_init(smem_u32(&sh.qempty[i]), 2);
+        }
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&sh.tfull[i]), 1);
             mbar_init(smem_u32(&sh.tempty[i]), 256);
-            mbar_init(smem_u32(&sh.qfull[i]), 1);
-            mbar_init(smem_u32(&sh.qempty[i]), 2);
             mbar_init(smem_u32(&sh.pub_full[i]), kFuEpiWarps * 32);
             for (int q = 0; q < 4; ++q) mbar_init(smem_u32(&sh.pbar[i][q]), 64);
         }
@@ -482,8 +501,8 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             const uint64_t pol_b = l2_policy_evict_first();    // second read: last use
             const uint64_t pol_q = l2_policy_evict_last();
             FuIter it(g, fa);
-            int q_phase = -1, vq[2] = {0, 0}, pending_rel = 0, b_idx = -1;
-            bool q_used[2] = {false, false};
+            int q_phase = -1, vq[kFuQBufs] = {0, 0, 0}, pending_rel = 0, b_idx = -1;
+            bool q_used[kFuQBufs] = {false, false, false};
             // next step of the list with everything the other roles need folded into its flags
             auto fetch = [&](FuPStep& e) -> bool {
                 while (true) {
@@ -492,17 +511,19 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     if (op.kind == kOpStop) return false;
                     if (op.kind == kOpPairEnd) {
                         // the query block of phase (pair - 1) has seen its last product
-                        const int b = (op.pair - 1) & 1;
-                        if (op.pair >= 1 && q_used[b]) {
-                            pending_rel |= b ? kStepRel1 : kStepRel0;
-                            q_used[b] = false;
+                        if (op.pair >= 1) {
+                            const int b = (op.pair - 1) % kFuQBufs;
+                            if (q_used[b]) {
+                                pending_rel |= 1 << (kStepRelShift + b);
+                                q_used[b] = false;
+                            }
                         }
                         if (it.pb.n_tiles > 0) ++b_idx;        // the new pair's sweep B phase needs the next fetch
                         continue;
                     }
                     const FuPhase& ph = op.kind == kOpA ? it.pa : it.pb;
-                    const int b = ph.phase & 1;
-                    int flags = pending_rel | (op.k << kStepKShift) | (b ? kStepQBuf : 0);
+                    const int b = ph.phase % kFuQBufs;
+                    int flags = pending_rel | (op.k << kStepKShift) | (b << kStepQBufShift);
                     pending_rel = 0;
                     e.qseq = -1;
                     if (op.kind == kOpA) {
@@ -522,9 +543,41 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     }
                     if ((vq[b] - 1) & 1) flags |= kStepQPar;
                     e.rec = make_int4(flags, op.tile * kTcTile, ph.Tn, ph.layer * g.total_tokens + ph.tok_base);
-                    e.j = ph.j; e.layer = ph.layer; e.prob = ph.prob; e.tok_row = ph.tok_base + op.tile * kTcTile;
+                    e.j = ph.j; e.layer = ph.layer; e.prob = ph.prob; e.tok_row = ph.tok_base + op.tile * kTcTile; e.phase = ph.phase;
                     return true;
                 }
+            };
+            // Query blocks are loaded a phase ahead of their first use: phase p goes to buffer p % 3
+            // as soon as that buffer's previous tenant (phase p - 3) has seen its last product.
+            int ql_phase = 0, ql_count[kFuQBufs] = {0, 0, 0}, ql_prob = it.group, ql_j = 0;
+            bool ql_tiles = false;
+            auto ql_problem = [&]() {                           // does this CTA hold tiles of problem ql_prob
+                const int seq = ql_prob % g.n_seqs, L = geo_L(g, seq);
+                ql_tiles = L > g.n_out && it.rank < (L + kTcTile - 1) / kTcTile;
+            };
+            ql_problem();
+            auto load_q = [&](int upto_phase, bool blocking) -> bool {
+                while (ql_phase < it.n_phases && ql_phase <= upto_phase) {
+                    if (ql_tiles) {
+                        const int b = ql_phase % kFuQBufs;
+                        if (ql_count[b] > 0) {
+                            const uint32_t par = (uint32_t)((ql_count[b] - 1) & 1);
+                            if (blocking) {
+                                if (!FU_WAIT(1, mbar_wait(smem_u32(&sh.qempty[b]), par, abort_flag))) return false;
+                            } else if (!mbar_try_wait(smem_u32(&sh.qempty[b]), par)) {
+                                return true;
+                            }
+                        }
+                        ++ql_count[b];
+                        mbar_expect_tx(smem_u32(&sh.qfull[b]), kFuTileBytes);
+                        for (int a = 0; a < 2; ++a)
+                            tma_load_2d(q_smem + b * kFuTileBytes + a * kAtomBytes, &tmQ, smem_u32(&sh.qfull[b]), a * 64,
+                                        ql_prob * g.H * g.window + ql_j * R, pol_q);
+                    }
+                    ++ql_phase;
+                    if (++ql_j == g.Hkv) { ql_j = 0; ql_prob += it.n_groups; if (ql_phase < it.n_phases) ql_problem(); }
+                }
+                return true;
             };
             FuPStep cur, nxt;
             bool have = fetch(cur);
@@ -534,14 +587,9 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 if (more) cur.rec.x |= kStepMore;
                 sched_post(sched, n_steps, cur.rec);
                 const bool is_b = (cur.rec.x & kStepB) != 0;
-                if (cur.qseq >= 0) {
-                    const int b = (cur.rec.x & kStepQBuf) ? 1 : 0;
-                    if (cur.qseq > 0 && !FU_WAIT(1, mbar_wait(smem_u32(&sh.qempty[b]), (cur.qseq - 1) & 1, abort_flag))) break;
-                    mbar_expect_tx(smem_u32(&sh.qfull[b]), kFuTileBytes);
-                    for (int a = 0; a < 2; ++a)
-                        tma_load_2d(q_smem + b * kFuTileBytes + a * kAtomBytes, &tmQ, smem_u32(&sh.qfull[b]), a * 64,
-                                    cur.prob * g.H * g.window + cur.j * R, pol_q);
-                }
+                // this step's query block must be on its way; the next phase's is started if its buffer is free
+                if (!load_q(cur.phase, true)) break;
+                load_q(cur.phase + 1, false);
                 const int st = n_steps % kFuStages, par = (n_steps / kFuStages) & 1;
                 FU_TRACE(0, n_steps, 0);
                 if (!FU_WAIT(2, mbar_wait(smem_u32(&sh.empty[st]), par ^ 1, abort_flag))) break;
@@ -562,13 +610,14 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         // wait for its barriers and read its next step while the other's products run.
         if (lane == 0) {
             const int acc = warp == 1 ? 0 : 1;
-            int n = 0, n_mine = 0, q_gen[2] = {0, 0}, q_seen[2] = {0, 0};
+            int n = 0, n_mine = 0, q_gen[kFuQBufs] = {0, 0, 0}, q_seen[kFuQBufs] = {0, 0, 0};
             int4 e;
             while (sched_get(sched, n, e, abort_flag)) {
                 const int flags = e.x;
-                if (flags & kStepRel0) tc_commit(smem_u32(&sh.qempty[0]));
-                if (flags & kStepRel1) tc_commit(smem_u32(&sh.qempty[1]));
-                const int b = (flags & kStepQBuf) ? 1 : 0;
+#pragma unroll
+                for (int i = 0; i < kFuQBufs; ++i)
+                    if (flags & (1 << (kStepRelShift + i))) tc_commit(smem_u32(&sh.qempty[i]));
+                const int b = (flags >> kStepQBufShift) & 3;
                 if (flags & kStepNewQ) ++q_gen[b];
                 const bool mine = (n & 1) == acc;
                 const int st = n % kFuStages, par = (n / kFuStages) & 1;
@@ -732,7 +781,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     tmem_ld32_issue(acc_addr + half * 64 + 32, r1);
                     tmem_ld_wait();
                     tc_fence_before();
-                    mbar_arrive(smem_u32(&sh.tempty[set]));        // logits are in registers: release the accumulator
+                    if (kReleaseAt == 0) mbar_arrive(smem_u32(&sh.tempty[set]));   // logits are in registers
                     if (first_thread) FU_TRACE(2 + set, n_mine, 2);
                     if (flags & kStepMask) {
                         const int tok0 = e.y + half * 64;
@@ -741,7 +790,9 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         chunk_mask(r1, tok0 + 32, lim);
                     }
                     rs.add(r0, c2);
+                    if (kReleaseAt == 1) mbar_arrive(smem_u32(&sh.tempty[set]));
                     rs.add(r1, c2);
+                    if (kReleaseAt == 2) mbar_arrive(smem_u32(&sh.tempty[set]));
                     if (first_thread) FU_TRACE(2 + set, n_mine, 3);
                     ++n_mine;
                 }
@@ -784,12 +835,14 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     tmem_ld16_issue(acc_addr + 96 + half * 16, v3);
                     tmem_ld_wait();
                     tc_fence_before();
-                    mbar_arrive(smem_u32(&sh.tempty[set]));
+                    if (kReleaseAt == 0) mbar_arrive(smem_u32(&sh.tempty[set]));
                     if (first_thread) FU_TRACE(2 + set, n_mine, 2);
                     accumulate_head16(accw, v0, lj, c2);
                     accumulate_head16(accw, v1, lj + 32, c2);
+                    if (kReleaseAt == 1) mbar_arrive(smem_u32(&sh.tempty[set]));
                     accumulate_head16(accw, v2, lj + 64, c2);
                     accumulate_head16(accw, v3, lj + 96, c2);
+                    if (kReleaseAt == 2) mbar_arrive(smem_u32(&sh.tempty[set]));
                     // \bar A of this token tile, summed over the KV heads seen so far
                     const uint32_t abar_addr = lane_addr + (uint32_t)(kFuAbarCol0 + ((flags >> kStepKShift) & 7) * 32 + half * 16);
                     if (!(flags & kStepHead0)) {
