@@ -44,6 +44,10 @@ constexpr int kFuMaxTilesPerCta = 7;         // \bar A slots in tensor memory: 7
 constexpr int kFuAbarCol0 = 256;             // columns [0, 256): two logit accumulators
 constexpr int kFuTmemCols = 512;
 constexpr int kFuLead = 2;                   // sweep A runs at least this many tiles ahead of sweep B
+#ifndef SABLOCK_RUN_AHEAD
+#define SABLOCK_RUN_AHEAD 0
+#endif
+constexpr int kFuRunAhead = SABLOCK_RUN_AHEAD;
 constexpr int kFuPartSlots = 4;              // ring of per-phase partial buffers in global memory
 constexpr int kFuLseSlots = 4;               // ring of log-sum-exp buffers in shared memory
 constexpr int kFuMaxCtasDev = 256;           // upper bound on the CTAs of one launch
@@ -76,10 +80,11 @@ struct FusedArgs {
 
 // Optional cycle-stamp trace of a few CTAs (compiled in with -DSABLOCK_TRACE; off otherwise):
 // role 0 = producer, 1 = MMA issuers (per step), 2 / 3 = first thread of epilogue set 0 / 1
-// (per own step).
+// (per own step), 4 / 5 = hand-over warp per phase (4: row sums taken, published, all CTAs in,
+// merged; 5: merges of all CTAs in, log-sum-exps fetched).
 #ifdef SABLOCK_TRACE
 constexpr int kTraceOps = 600;
-__device__ long long g_trace[4][4][kTraceOps][4];   // [traced CTA][role][step][event]
+__device__ long long g_trace[4][6][kTraceOps][4];   // [traced CTA][role][step][event]
 #define FU_TRACE(role, n, ev)                                                                 \
     do {                                                                                      \
         if (tslot >= 0 && (n) < kTraceOps) g_trace[tslot][role][n][ev] = clock64();           \
@@ -107,91 +112,100 @@ enum { kOpA = 0, kOpB = 1, kOpPairEnd = 2, kOpStop = 3 };
 
 // What the producer needs to know about one phase = (problem, KV head).
 struct FuPhase {
-    int phase;       // phase counter of the group; -1 = none
     int prob, j;     // problem index and KV head
     int layer;
     int Tn;          // compressible length of the sequence
     int tok_base;    // first packed token row of the sequence
-    int n_tiles;     // tiles of this CTA in the sweep in question
+    int n_a, n_b;    // tiles of this CTA in sweep A and in sweep B
+    int qpar;        // parity of the load of this phase's query block into its buffer
 };
 
 struct FuOp {
     int kind;
+    int phase;
     int k;           // which of the CTA's tiles (slot of \bar A in tensor memory)
     int tile;        // token tile index inside the sequence
     int last;        // last tile of this kind for this CTA in this phase
-    int pair;        // the pair this step belongs to (for kOpPairEnd: the pair that ended)
+    int released;    // kOpPairEnd: the query-block buffer of the phase whose sweep B just ended, or -1
 };
 
-// Walk over the work list of one CTA (run by the producer thread only).  Pair n holds the sweep A
-// tiles of phase n (`pa`) and the sweep B tiles of phase n - 1 (`pb`); all divisions happen when a
-// pair begins.  Inside a pair sweep A leads by at least kFuLead tiles, and by more while the
-// log-sum-exps of phase n - 1 are not in yet (`b_ready` false).
+// Walk over the work list of one CTA (run by the producer thread only) with two cursors: sweep A
+// at phase `a_ph`, sweep B behind it at phase `b_ph` < a_ph.  Normally sweep B follows one phase
+// behind and sweep A leads by at least kFuLead tiles inside that phase.  While the log-sum-exps of
+// sweep B's phase are not in yet (`b_ready` false: another CTA is late) sweep A simply runs on,
+// up to two phases ahead (three query-block buffers), instead of idling; the second read of K then
+// comes a little later, which costs L2 hits only while it lasts.
 struct FuIter {
     const Geo& g;
     int cpp, n_groups, group, rank;
     int n_phases;            // phases of this group
-    int pair, ia, ib;
-    int tiles_b;             // sweep B tiles of this CTA in pa's problem
-    FuPhase pa, pb;
+    int a_ph, ia, b_ph, ib;
+    int a_buf, b_buf;        // a_ph % 3 and b_ph % 3 (query-block buffers), kept without divisions
+    FuPhase pa;              // phase a_ph
+    FuPhase q0, q1;          // phases b_ph and b_ph + 1 where those lie behind sweep A
     __device__ FuIter(const Geo& geo, const FusedArgs& a) : g(geo), cpp(a.cpp), n_groups(a.n_groups)
     {
         group = blockIdx.x / cpp;
         rank = blockIdx.x % cpp;
         const int my_probs = group < n_groups ? (a.n_prob - group + n_groups - 1) / n_groups : 0;
         n_phases = my_probs * g.Hkv;
-        pair = 0; ia = ib = 0; tiles_b = 0;
-        pb.phase = -1; pb.n_tiles = 0;
-        pa.j = 0; pa.prob = group; pa.n_tiles = 0;
-        load_a();
+        a_ph = ia = b_ph = ib = a_buf = b_buf = 0;
+        pa.prob = group; pa.j = -1; pa.n_a = pa.n_b = 0;
+        if (n_phases > 0) load_next();
     }
     __device__ int my_tiles(int n) const { return rank < n ? (n - rank + cpp - 1) / cpp : 0; }
-    // Phase `pair` for sweep A.  Consecutive phases of a problem differ only in the KV head; the
-    // divisions are paid once per problem.
-    __device__ void load_a()
+    // Turns pa into the next phase.  Consecutive phases of a problem differ only in the KV head;
+    // the divisions are paid once per problem.
+    __device__ void load_next()
     {
-        pa.phase = pair;
-        if (pair >= n_phases) { pa.phase = -1; pa.n_tiles = 0; return; }
-        if (pair > 0 && pa.j + 1 < g.Hkv) { ++pa.j; return; }           // same problem, next KV head
-        pa.prob = pair == 0 ? group : pa.prob + n_groups;
+        if (pa.j >= 0 && pa.j + 1 < g.Hkv) { ++pa.j; return; }
+        if (pa.j >= 0) pa.prob += n_groups;
         pa.j = 0;
         pa.layer = pa.prob / g.n_seqs;
         const int seq = pa.prob - pa.layer * g.n_seqs;
         pa.tok_base = g.cu[seq];
         const int L = g.cu[seq + 1] - pa.tok_base;
         pa.Tn = L - g.window;
-        pa.n_tiles = L > g.n_out ? my_tiles((L + kTcTile - 1) / kTcTile) : 0;   // else: returned unchanged
-        tiles_b = pa.n_tiles > 0 ? my_tiles((pa.Tn + kTcTile - 1) / kTcTile) : 0;
+        pa.n_a = L > g.n_out ? my_tiles((L + kTcTile - 1) / kTcTile) : 0;       // else: returned unchanged
+        pa.n_b = pa.n_a > 0 ? my_tiles((pa.Tn + kTcTile - 1) / kTcTile) : 0;
     }
-    __device__ void next_pair()
-    {
-        pb = pa;
-        pb.n_tiles = pa.phase >= 0 ? tiles_b : 0;
-        ++pair; ia = ib = 0;
-        load_a();
-    }
-    __device__ bool b_pending() const { return ib < pb.n_tiles; }
+    __device__ bool b_pending() const { return b_ph < a_ph && ib < q0.n_b; }
     __device__ FuOp next(bool b_ready)
     {
         FuOp op;
-        op.pair = pair;
-        if (pair > n_phases) { op.kind = kOpStop; return op; }
-        const bool can_a = ia < pa.n_tiles, can_b = ib < pb.n_tiles;
-        const bool take_a = can_a && (!can_b || ia < ib + kFuLead || !b_ready);
-        if (take_a) {
-            op.kind = kOpA; op.k = ia; op.last = ia == pa.n_tiles - 1;
+        op.released = -1;
+        // sweep B leaves a phase when its tiles are done (at once if it has none)
+        if (b_ph < a_ph && ib >= q0.n_b) {
+            op.kind = kOpPairEnd;
+            op.released = q0.n_a > 0 ? b_buf : -1;
+            q0 = q1;
+            ++b_ph; ib = 0;
+            b_buf = b_buf == kFuQBufs - 1 ? 0 : b_buf + 1;
+            return op;
+        }
+        // sweep A moves on to the next phase when its tiles are done and a buffer is free for it
+        if (a_ph < n_phases && ia >= pa.n_a && a_ph + 1 <= b_ph + kFuQBufs - 1) {
+            if (a_ph == b_ph) q0 = pa; else q1 = pa;
+            ++a_ph; ia = 0;
+            a_buf = a_buf == kFuQBufs - 1 ? 0 : a_buf + 1;
+            if (a_ph < n_phases) load_next();
+            op.kind = kOpPairEnd;
+            return op;
+        }
+        // how far sweep A may run into the phase after next (in tiles) while sweep B waits
+        const bool can_a = a_ph < n_phases && ia < pa.n_a && (a_ph <= b_ph + 1 || ia < kFuRunAhead);
+        const bool can_b = b_ph < a_ph && ib < q0.n_b;
+        if (!can_a && !can_b) { op.kind = kOpStop; return op; }
+        const bool lead_needed = a_ph == b_ph + 1 && ia < ib + kFuLead;
+        if (can_a && (!can_b || !b_ready || lead_needed)) {
+            op.kind = kOpA; op.phase = a_ph; op.k = ia; op.last = ia == pa.n_a - 1;
             op.tile = rank + ia * cpp;
             ++ia;
             return op;
         }
-        if (can_b) {
-            op.kind = kOpB; op.k = ib; op.last = ib == pb.n_tiles - 1;
-            op.tile = rank + ib * cpp;
-            ++ib;
-            return op;
-        }
-        op.kind = kOpPairEnd;
-        next_pair();
+        op.kind = kOpB; op.phase = b_ph; op.k = ib; op.last = ib == q0.n_b - 1;
+        op.tile = rank + ib * cpp;
+        ++ib;
         return op;
     }
 };
@@ -199,7 +213,6 @@ struct FuIter {
 // One tile step as the other roles see it: 16 bytes in the shared-memory ring.
 constexpr int kStepB = 1 << 0;          // sweep B (else sweep A)
 constexpr int kStepLastA = 1 << 1;      // last sweep A step of its phase for this CTA: row sums are due
-constexpr int kStepMore = 1 << 2;       // another step follows
 constexpr int kStepFirstB = 1 << 3;     // first sweep B step of its phase for this CTA: next log-sum-exp buffer
 constexpr int kStepKShift = 4;          // bits 4-6: slot of the tile among the CTA's tiles
 constexpr int kStepHead0 = 1 << 7;      // first KV head of the layer (sweep B starts \bar A afresh)
@@ -433,12 +446,6 @@ __device__ __forceinline__ void accumulate_head16(float (&accw)[16], const uint3
     }
 }
 
-// A step as the producer holds it before posting.
-struct FuPStep {
-    int4 rec;
-    int j, layer, prob, tok_row, qseq, phase;
-};
-
 __global__ void __launch_bounds__(kFuThreads, 1)
 score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const Geo g,
                const FusedArgs fa)
@@ -501,106 +508,97 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             const uint64_t pol_b = l2_policy_evict_first();    // second read: last use
             const uint64_t pol_q = l2_policy_evict_last();
             FuIter it(g, fa);
-            int q_phase = -1, vq[kFuQBufs] = {0, 0, 0}, pending_rel = 0, b_idx = -1;
-            bool q_used[kFuQBufs] = {false, false, false};
-            // next step of the list with everything the other roles need folded into its flags
-            auto fetch = [&](FuPStep& e) -> bool {
-                while (true) {
-                    const bool b_ready = sched.lse_fetched > b_idx;
-                    const FuOp op = it.next(b_ready);
-                    if (op.kind == kOpStop) return false;
-                    if (op.kind == kOpPairEnd) {
-                        // the query block of phase (pair - 1) has seen its last product
-                        if (op.pair >= 1) {
-                            const int b = (op.pair - 1) % kFuQBufs;
-                            if (q_used[b]) {
-                                pending_rel |= 1 << (kStepRelShift + b);
-                                q_used[b] = false;
-                            }
-                        }
-                        if (it.pb.n_tiles > 0) ++b_idx;        // the new pair's sweep B phase needs the next fetch
-                        continue;
-                    }
-                    const FuPhase& ph = op.kind == kOpA ? it.pa : it.pb;
-                    const int b = ph.phase % kFuQBufs;
-                    int flags = pending_rel | (op.k << kStepKShift) | (b << kStepQBufShift);
-                    pending_rel = 0;
-                    e.qseq = -1;
-                    if (op.kind == kOpA) {
-                        if (op.last) flags |= kStepLastA;
-                        if (op.tile * kTcTile + kTcTile - 1 > ph.Tn) flags |= kStepMask;
-                        if (ph.phase != q_phase) {             // first tile of a phase: its query block
-                            q_phase = ph.phase;
-                            e.qseq = vq[b]++;
-                            q_used[b] = true;
-                            flags |= kStepNewQ;
-                        }
-                    } else {
-                        flags |= kStepB;
-                        if (op.k == 0) flags |= kStepFirstB;
-                        if (ph.j == 0) flags |= kStepHead0;
-                        if (ph.j == g.Hkv - 1) flags |= kStepHeadLast;
-                    }
-                    if ((vq[b] - 1) & 1) flags |= kStepQPar;
-                    e.rec = make_int4(flags, op.tile * kTcTile, ph.Tn, ph.layer * g.total_tokens + ph.tok_base);
-                    e.j = ph.j; e.layer = ph.layer; e.prob = ph.prob; e.tok_row = ph.tok_base + op.tile * kTcTile; e.phase = ph.phase;
-                    return true;
-                }
-            };
             // Query blocks are loaded a phase ahead of their first use: phase p goes to buffer p % 3
             // as soon as that buffer's previous tenant (phase p - 3) has seen its last product.
-            int ql_phase = 0, ql_count[kFuQBufs] = {0, 0, 0}, ql_prob = it.group, ql_j = 0;
+            int ql_phase = 0, ql_buf = 0, ql_prob = it.group, ql_j = 0;
+            unsigned ql_used = 0, ql_par = 0;                  // per buffer: ever loaded, parity of its load count
             bool ql_tiles = false;
-            auto ql_problem = [&]() {                           // does this CTA hold tiles of problem ql_prob
+            {
                 const int seq = ql_prob % g.n_seqs, L = geo_L(g, seq);
-                ql_tiles = L > g.n_out && it.rank < (L + kTcTile - 1) / kTcTile;
-            };
-            ql_problem();
-            auto load_q = [&](int upto_phase, bool blocking) -> bool {
-                while (ql_phase < it.n_phases && ql_phase <= upto_phase) {
+                ql_tiles = it.n_phases > 0 && L > g.n_out && it.rank < (L + kTcTile - 1) / kTcTile;
+            }
+            unsigned fq_par = 0;                               // the same parities as the work list sees them
+            int q_phase = -1, pending_rel = 0, b_idx = -1, b_counted = -1, n_steps = 0;
+            bool ok = true;
+            while (ok) {
+                // ---- next step of the work list
+                if (it.b_pending() && b_counted != it.b_ph) {  // sweep B entered a phase: it needs the helper's next fetch
+                    b_counted = it.b_ph;
+                    ++b_idx;
+                }
+                const FuOp op = it.next(sched.lse_fetched > b_idx);
+                if (op.kind == kOpStop) break;
+                if (op.kind == kOpPairEnd) {
+                    // the query block of a phase whose sweep B ended has seen its last product
+                    if (op.released >= 0) pending_rel |= 1 << (kStepRelShift + op.released);
+                    continue;
+                }
+                const bool is_b = op.kind == kOpB;
+                FuPhase& ph = is_b ? it.q0 : it.pa;
+                const int b = is_b ? it.b_buf : it.a_buf;
+                int flags = pending_rel | (op.k << kStepKShift) | (b << kStepQBufShift);
+                pending_rel = 0;
+                if (!is_b) {
+                    if (op.last) flags |= kStepLastA;
+                    if (op.tile * kTcTile + kTcTile - 1 > ph.Tn) flags |= kStepMask;
+                    if (op.phase != q_phase) {                 // first tile of a phase: its query block
+                        q_phase = op.phase;
+                        ph.qpar = (fq_par >> b) & 1;
+                        fq_par ^= 1u << b;
+                        flags |= kStepNewQ;
+                    }
+                } else {
+                    flags |= kStepB;
+                    if (op.k == 0) flags |= kStepFirstB;
+                    if (ph.j == 0) flags |= kStepHead0;
+                    if (ph.j == g.Hkv - 1) flags |= kStepHeadLast;
+                }
+                if (ph.qpar) flags |= kStepQPar;
+                const int tok0 = op.tile * kTcTile;
+                sched_post(sched, n_steps, make_int4(flags, tok0, ph.Tn, ph.layer * g.total_tokens + ph.tok_base));
+                FU_TRACE(0, n_steps, 3);
+                // ---- query blocks: this step's must be on its way (blocking); the next phase's is
+                // started if its buffer is free (probe only)
+                while (ql_phase < it.n_phases && ql_phase <= op.phase + 1) {
                     if (ql_tiles) {
-                        const int b = ql_phase % kFuQBufs;
-                        if (ql_count[b] > 0) {
-                            const uint32_t par = (uint32_t)((ql_count[b] - 1) & 1);
-                            if (blocking) {
-                                if (!FU_WAIT(1, mbar_wait(smem_u32(&sh.qempty[b]), par, abort_flag))) return false;
-                            } else if (!mbar_try_wait(smem_u32(&sh.qempty[b]), par)) {
-                                return true;
+                        if ((ql_used >> ql_buf) & 1) {
+                            const uint32_t par = ((ql_par >> ql_buf) & 1) ^ 1;
+                            if (ql_phase <= op.phase) {
+                                if (!FU_WAIT(1, mbar_wait(smem_u32(&sh.qempty[ql_buf]), par, abort_flag))) { ok = false; break; }
+                            } else if (!mbar_test_wait(smem_u32(&sh.qempty[ql_buf]), par)) {
+                                break;
                             }
                         }
-                        ++ql_count[b];
-                        mbar_expect_tx(smem_u32(&sh.qfull[b]), kFuTileBytes);
+                        ql_used |= 1u << ql_buf;
+                        ql_par ^= 1u << ql_buf;
+                        mbar_expect_tx(smem_u32(&sh.qfull[ql_buf]), kFuTileBytes);
                         for (int a = 0; a < 2; ++a)
-                            tma_load_2d(q_smem + b * kFuTileBytes + a * kAtomBytes, &tmQ, smem_u32(&sh.qfull[b]), a * 64,
+                            tma_load_2d(q_smem + ql_buf * kFuTileBytes + a * kAtomBytes, &tmQ, smem_u32(&sh.qfull[ql_buf]), a * 64,
                                         ql_prob * g.H * g.window + ql_j * R, pol_q);
                     }
                     ++ql_phase;
-                    if (++ql_j == g.Hkv) { ql_j = 0; ql_prob += it.n_groups; if (ql_phase < it.n_phases) ql_problem(); }
+                    ql_buf = ql_buf == kFuQBufs - 1 ? 0 : ql_buf + 1;
+                    if (++ql_j == g.Hkv) {
+                        ql_j = 0;
+                        ql_prob += it.n_groups;
+                        if (ql_phase < it.n_phases) {
+                            const int seq = ql_prob % g.n_seqs, L = geo_L(g, seq);
+                            ql_tiles = L > g.n_out && it.rank < (L + kTcTile - 1) / kTcTile;
+                        }
+                    }
                 }
-                return true;
-            };
-            FuPStep cur, nxt;
-            bool have = fetch(cur);
-            int n_steps = 0;
-            while (have) {
-                const bool more = fetch(nxt);
-                if (more) cur.rec.x |= kStepMore;
-                sched_post(sched, n_steps, cur.rec);
-                const bool is_b = (cur.rec.x & kStepB) != 0;
-                // this step's query block must be on its way; the next phase's is started if its buffer is free
-                if (!load_q(cur.phase, true)) break;
-                load_q(cur.phase + 1, false);
+                if (!ok) break;
+                // ---- the K tile of the step
                 const int st = n_steps % kFuStages, par = (n_steps / kFuStages) & 1;
                 FU_TRACE(0, n_steps, 0);
                 if (!FU_WAIT(2, mbar_wait(smem_u32(&sh.empty[st]), par ^ 1, abort_flag))) break;
                 FU_TRACE(0, n_steps, 1);
                 mbar_expect_tx(smem_u32(&sh.full[st]), kFuTileBytes);
                 for (int a = 0; a < 2; ++a)
-                    tma_load_4d(k_smem + st * kFuTileBytes + a * kAtomBytes, &tmK, smem_u32(&sh.full[st]), a * 64, cur.j,
-                                cur.tok_row, cur.layer, is_b ? pol_b : pol_a);
+                    tma_load_4d(k_smem + st * kFuTileBytes + a * kAtomBytes, &tmK, smem_u32(&sh.full[st]), a * 64, ph.j,
+                                ph.tok_base + tok0, ph.layer, is_b ? pol_b : pol_a);
+                FU_TRACE(0, n_steps, 2);
                 ++n_steps;
-                cur = nxt;
-                have = more;
             }
             sched.final_ = 1;
         }
@@ -641,7 +639,6 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     ++n_mine;
                 }
                 ++n;
-                if (!(flags & kStepMore)) break;
             }
         }
     } else if (warp == kFuHelpWarp) {
@@ -672,6 +669,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 if (!ok) break;
                 const int buf = n_pub & 1;
                 if (!FU_WAIT(6, mbar_wait(smem_u32(&sh.pub_full[buf]), (uint32_t)((n_pub >> 1) & 1), abort_flag))) break;
+                if (lane == 0) FU_TRACE(4, phase, 0);
                 float2* dst = fa.part + (((size_t)group * kFuPartSlots + (phase % kFuPartSlots)) * fa.cpp + rank) * R;
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
@@ -696,12 +694,14 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 if (lane == 0) {
                     sched.pub_done = n_pub;
                     atomicAdd(fa.arrive + prob * g.Hkv + j, 1);
+                    FU_TRACE(4, phase, 1);
                 }
             }
             if (rank < R) {
                 if (lane == 0) ok = FU_WAIT(12, wait_counter(fa.arrive + prob * g.Hkv + j, n_src, abort_flag, fa.status));
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
+                if (lane == 0) FU_TRACE(4, phase, 2);
                 const float2* pp = fa.part + ((size_t)group * kFuPartSlots + (phase % kFuPartSlots)) * fa.cpp * R;
                 for (int row = rank; row < R; row += fa.cpp) {
                     // one partial per source CTA, merged in index order; all loads of a lane are issued
@@ -730,6 +730,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 if (lane == 0) {
                     __threadfence();
                     atomicAdd(fa.done + prob * g.Hkv + j, 1);
+                    FU_TRACE(4, phase, 3);
                 }
             }
             // the finished log-sum-exps, if this CTA runs sweep B for the phase
@@ -737,6 +738,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 if (lane == 0) ok = FU_WAIT(13, wait_counter(fa.done + prob * g.Hkv + j, n_mergers, abort_flag, fa.status));
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
+                if (lane == 0) FU_TRACE(5, phase, 0);
                 const int slot = n_fetch % kFuLseSlots;
                 const float* src = fa.lse2 + (size_t)prob * g.H * g.window + j * R;
 #pragma unroll
@@ -746,6 +748,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 if (lane == 0) {
                     mbar_arrive(smem_u32(&sh.lse_full[slot]));
                     sched.lse_fetched = n_fetch;
+                    FU_TRACE(5, phase, 1);
                 }
             }
         }
@@ -887,7 +890,6 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     ++n_mine;
                 }
             }
-            if (!(flags & kStepMore)) break;
         }
     }
 
