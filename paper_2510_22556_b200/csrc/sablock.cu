@@ -62,7 +62,7 @@ struct Plan {
     int n_chunks;              // pass-1 partials per row
     int keep_words, long_cap, seg_tiles;
     // workspace offsets
-    size_t o_status, o_ticket, o_long_count, o_tile_state, o_keep, o_arrive, o_done, control_bytes;
+    size_t o_status, o_ticket, o_long_count, o_tile_state, o_keep, o_arrive, o_done, o_top, control_bytes;
     size_t o_seg_id, o_seg_start, o_n_seg, o_s_raw, o_s, o_e, o_sr, o_part, o_lse, o_thr, o_cut, o_long_list,
         o_phi, o_rank, o_fpart, total;
 };
@@ -196,6 +196,7 @@ sablock_status_t make_plan(const sablock_params_t* p, int n_layers, int n_seqs, 
     pl->o_keep = take(sizeof(unsigned) * (size_t)pl->n_prob * pl->keep_words);
     pl->o_arrive = take(sizeof(int) * (size_t)pl->n_prob * g.Hkv);
     pl->o_done = take(sizeof(int) * (size_t)pl->n_prob * g.Hkv);
+    pl->o_top = take(sizeof(TopScratch) * (size_t)pl->n_prob);
     pl->control_bytes = o;
     const size_t ntok = (size_t)n_layers * total_tokens;
     pl->o_seg_id = take(sizeof(int) * total_tokens);
@@ -446,8 +447,35 @@ sablock_status_t run_select(const Plan& pl, const sablock_params_t* p, const flo
     const Geo& g = pl.geo;
     unsigned* thr = at<unsigned>(ws, pl.o_thr);
     int* cut = at<int>(ws, pl.o_cut);
-    topb_kernel<<<pl.n_prob, kTopThreads, 0, stream>>>(g, s_ref, thr, cut);
-    SAB_TRY(check_launch());
+    {
+        // Several CTAs per problem when the problems are few and long; they wait for one another,
+        // hence the cooperative launch (all CTAs co-resident or an error).
+        int ctas = 1;
+        int dev = 0, sms = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0) {
+            ctas = sms / pl.n_prob;
+            const int by_len = (pl.max_L + 4 * kTopThreads - 1) / (4 * kTopThreads);      // at least four rounds each
+            if (ctas > by_len) ctas = by_len;
+            if (ctas > kTopMaxCtas) ctas = kTopMaxCtas;
+            if (ctas < 1) ctas = 1;
+        }
+        TopScratch* tsc = at<TopScratch>(ws, pl.o_top);
+        int* status = at<int>(ws, pl.o_status);
+        if (ctas > 1) {
+            Geo geo = g;
+            const float* sr = s_ref;
+            void* args[] = {&geo, &sr, &thr, &cut, &tsc, &status};
+            if (cudaLaunchCooperativeKernel((const void*)topb_kernel, dim3(ctas, pl.n_prob), dim3(kTopThreads), args, 0, stream) !=
+                cudaSuccess) {
+                cudaGetLastError();
+                return SABLOCK_ERR_CUDA;
+            }
+            ++t_launches;
+        } else {
+            topb_kernel<<<dim3(1, pl.n_prob), kTopThreads, 0, stream>>>(g, s_ref, thr, cut, tsc, status);
+            SAB_TRY(check_launch());
+        }
+    }
     prof_mark(5, stream);
     SearchOut so;
     so.keep = at<unsigned>(ws, pl.o_keep);

@@ -214,20 +214,54 @@ __device__ __forceinline__ unsigned order_key(float f)
 }
 
 constexpr int kTopThreads = 1024;
+constexpr int kTopMaxCtas = 8;         // CTAs that may share one problem
 
-__global__ void __launch_bounds__(kTopThreads)
-topb_kernel(Geo g, const float* __restrict__ s_ref, unsigned* __restrict__ sel_thr, int* __restrict__ sel_cut)
+// Scratch of the multi-CTA select, per problem (zeroed before the launch).
+struct TopScratch {
+    int hist[4][256];                  // digit histograms of the four passes, summed over the CTAs
+    int arrived[5];                    // CTAs that have added their share (passes 0-3, tie count)
+    int eq_count[kTopMaxCtas];         // keys equal to the threshold in each CTA's slice
+};
+
+// Bounded wait until every CTA of the problem has contributed; false if it gave up.
+__device__ __forceinline__ bool top_wait(const int* ctr, int target, int* status)
 {
-    const int p = blockIdx.x, layer = p / g.n_seqs, seq = p % g.n_seqs;
+    const long long t0 = clock64();
+    while (true) {
+        int v;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ctr) : "memory");
+        if (v >= target) return true;
+        if (clock64() - t0 > 2000000000LL) {
+            atomicOr(status, kStatTimeout);
+            return false;
+        }
+        __nanosleep(100);
+    }
+}
+
+// grid = (ctas per problem, problems).  The CTAs of a problem each histogram a slice of the
+// scores and combine through integer atomics (sums of integers: the result does not depend on the
+// order), so all of them see the same digit counts and walk the same path.  The CTAs of a problem
+// wait for one another: the launch must keep them co-resident (the host launches cooperatively
+// when there is more than one per problem).
+__global__ void __launch_bounds__(kTopThreads)
+topb_kernel(Geo g, const float* __restrict__ s_ref, unsigned* __restrict__ sel_thr, int* __restrict__ sel_cut,
+            TopScratch* __restrict__ scratch, int* status)
+{
+    const int p = blockIdx.y, layer = p / g.n_seqs, seq = p % g.n_seqs;
     if (geo_identity(g, seq)) return;
     const int T = geo_L(g, seq) - g.window;
     const float* x = s_ref + (size_t)layer * g.total_tokens + g.cu[seq];
     const int tid = threadIdx.x, lane = tid & 31;
+    const int n_cta = gridDim.x, cta = blockIdx.x;
+    // this CTA's slice [a0, z0), a multiple of the block size long except for the last
+    const int per = ((T + n_cta - 1) / n_cta + kTopThreads - 1) / kTopThreads * kTopThreads;
+    const int a0 = min(cta * per, T), z0 = min(a0 + per, T);
+    TopScratch* sc = scratch + p;
     __shared__ int hist[256];
     __shared__ unsigned s_prefix;
-    __shared__ int s_k, s_neq;
+    __shared__ int s_k, s_neq, s_ok;
     __shared__ int s_scan[kTopThreads / 32];
-    __shared__ int s_cut;
 
     unsigned prefix = 0, mask = 0;
     int k = g.B;                                   // rank (1-based, descending) still to locate
@@ -236,18 +270,33 @@ topb_kernel(Geo g, const float* __restrict__ s_ref, unsigned* __restrict__ sel_t
         const int shift = 24 - 8 * pass;
         if (tid < 256) hist[tid] = 0;
         __syncthreads();
-        for (int i0 = 0; i0 < T; i0 += kTopThreads) {
+        for (int i0 = a0; i0 < z0; i0 += kTopThreads) {
             const int i = i0 + tid;
             int bin = 256;
-            if (i < T) {
+            if (i < z0) {
                 unsigned u = order_key(x[i]);
                 if ((u & mask) == prefix) bin = (u >> shift) & 255;
             }
             // one shared-memory atomic per distinct digit per warp
-            unsigned peers = __match_any_sync(0xffffffffu, bin);
-            if (bin < 256 && lane == __ffs(peers) - 1) atomicAdd(&hist[bin], __popc(peers));
+            if (__any_sync(0xffffffffu, bin < 256)) {
+                unsigned peers = __match_any_sync(0xffffffffu, bin);
+                if (bin < 256 && lane == __ffs(peers) - 1) atomicAdd(&hist[bin], __popc(peers));
+            }
         }
         __syncthreads();
+        if (n_cta > 1) {
+            if (tid < 256 && hist[tid]) atomicAdd(&sc->hist[pass][tid], hist[tid]);
+            __threadfence();
+            __syncthreads();
+            if (tid == 0) {
+                atomicAdd(&sc->arrived[pass], 1);
+                s_ok = top_wait(&sc->arrived[pass], n_cta, status) ? 1 : 0;
+            }
+            __syncthreads();
+            if (!s_ok) return;
+            if (tid < 256) hist[tid] = __ldcg(&sc->hist[pass][tid]);
+            __syncthreads();
+        }
         if (tid == 0) {
             int above = 0, d = 255;
             for (; d > 0; --d) {
@@ -268,8 +317,9 @@ topb_kernel(Geo g, const float* __restrict__ s_ref, unsigned* __restrict__ sel_t
     // k of the n_eq tokens whose key equals the threshold are taken, lowest indices first.
     int cut = T;                                   // all of them
     if (k < n_eq) {
-        const int chunk = (T + kTopThreads - 1) / kTopThreads;
-        const int a = tid * chunk, z = min(a + chunk, T);
+        const int len = z0 - a0;
+        const int chunk = (len + kTopThreads - 1) / kTopThreads;
+        const int a = a0 + tid * chunk, z = min(a + chunk, z0);
         int c = 0;
         for (int i = a; i < z; ++i) c += (order_key(x[i]) == prefix);
         int inc = c;
@@ -280,18 +330,33 @@ topb_kernel(Geo g, const float* __restrict__ s_ref, unsigned* __restrict__ sel_t
         }
         if (lane == 31) s_scan[tid >> 5] = inc;
         __syncthreads();
-        int woff = 0;
-        for (int w = 0; w < (tid >> 5); ++w) woff += s_scan[w];
-        const int excl = woff + inc - c;
-        if (excl < k && k <= excl + c) {
+        int woff = 0, total = 0;
+        for (int w = 0; w < kTopThreads / 32; ++w) {
+            if (w < (tid >> 5)) woff += s_scan[w];
+            total += s_scan[w];
+        }
+        int before = 0;                            // equal keys in the slices of the CTAs before this one
+        if (n_cta > 1) {
+            if (tid == 0) {
+                sc->eq_count[cta] = total;
+                __threadfence();
+                atomicAdd(&sc->arrived[4], 1);
+                s_ok = top_wait(&sc->arrived[4], n_cta, status) ? 1 : 0;
+            }
+            __syncthreads();
+            if (!s_ok) return;
+            for (int i = 0; i < cta; ++i) before += __ldcg(&sc->eq_count[i]);
+        }
+        const int excl = before + woff + inc - c;
+        if (excl < k && k <= excl + c) {           // the k-th equal key lies in this thread's chunk
             int seen = excl;
             for (int i = a; i < z; ++i)
-                if (order_key(x[i]) == prefix && ++seen == k) { s_cut = i; break; }
+                if (order_key(x[i]) == prefix && ++seen == k) { sel_cut[p] = i; break; }
         }
-        __syncthreads();
-        cut = s_cut;
+        if (cta == 0 && tid == 0) sel_thr[p] = prefix;
+        return;
     }
-    if (tid == 0) {
+    if (cta == 0 && tid == 0) {
         sel_thr[p] = prefix;
         sel_cut[p] = cut;
     }
