@@ -87,6 +87,9 @@ typedef struct sablock_params {
 void sablock_params_default(sablock_params_t *p);
 const char *sablock_status_string(sablock_status_t st);
 int sablock_version(void);
+/* Text of the most recent CUDA runtime error an entry point of this thread ran into (which call,
+ * after how many kernel launches of that entry point, and the runtime's message); "" if none. */
+const char *sablock_last_cuda_error(void);
 size_t sablock_params_sizeof(void);   /* sizeof(sablock_params_t) as the library was built */
 
 /* Bytes of device scratch needed for a call over n_layers x n_seqs problems whose

@@ -26,7 +26,7 @@ EXPORTS = [
     "sablock_read_status", "sablock_segment", "sablock_score", "sablock_select", "sablock_compact",
     "sablock_compress", "sablock_compress_layers", "sablock_compress_layers_host", "sablock_last_launch_count",
     "sablock_params_sizeof", "sablock_workspace_region", "sablock_profile_enable", "sablock_profile_read",
-    "sablock_profile_stage_name", "sablock_segment_static",
+    "sablock_profile_stage_name", "sablock_segment_static", "sablock_last_cuda_error",
 ]
 
 
@@ -46,7 +46,9 @@ class Params(C.Structure):
 class SablockError(RuntimeError):
     def __init__(self, code: int, where: str):
         self.code = code
-        super().__init__(f"{where}: {STATUS_NAMES.get(code, code)} ({lib().sablock_status_string(code).decode()})")
+        detail = lib().sablock_last_cuda_error().decode() if code == 4 else ""
+        super().__init__(f"{where}: {STATUS_NAMES.get(code, code)} ({lib().sablock_status_string(code).decode()})"
+                         + (f" [{detail}]" if detail else ""))
 
 
 _lib = None
@@ -61,6 +63,7 @@ def lib():
                               "or __graft_entry__.build()")
         l = C.CDLL(LIB_PATH)
         l.sablock_status_string.restype = C.c_char_p
+        l.sablock_last_cuda_error.restype = C.c_char_p
         l.sablock_params_sizeof.restype = C.c_size_t
         if l.sablock_params_sizeof() != C.sizeof(Params):
             raise ImportError("sablock_params_t layout mismatch between the library and the binding")

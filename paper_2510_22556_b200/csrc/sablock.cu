@@ -222,16 +222,27 @@ sablock_status_t make_plan(const sablock_params_t* p, int n_layers, int n_seqs, 
 
 template <typename T> T* at(void* ws, size_t off) { return reinterpret_cast<T*>(static_cast<char*>(ws) + off); }
 
+thread_local char t_cuda_error[160] = "";
+
+// Remembers what the CUDA runtime said, for sablock_last_cuda_error().
+sablock_status_t note_cuda_error(cudaError_t err, const char* where)
+{
+    snprintf(t_cuda_error, sizeof(t_cuda_error), "%s after launch %d: %s", where, t_launches, cudaGetErrorString(err));
+    return SABLOCK_ERR_CUDA;
+}
+
 sablock_status_t check_launch()
 {
     ++t_launches;
-    return cudaGetLastError() == cudaSuccess ? SABLOCK_OK : SABLOCK_ERR_CUDA;
+    const cudaError_t err = cudaGetLastError();
+    return err == cudaSuccess ? SABLOCK_OK : note_cuda_error(err, "kernel launch");
 }
 #define SAB_TRY(expr) do { sablock_status_t _s = (expr); if (_s != SABLOCK_OK) return _s; } while (0)
 
 sablock_status_t zero_control(const Plan& pl, void* ws, cudaStream_t stream)
 {
-    return cudaMemsetAsync(ws, 0, pl.control_bytes, stream) == cudaSuccess ? SABLOCK_OK : SABLOCK_ERR_CUDA;
+    const cudaError_t err = cudaMemsetAsync(ws, 0, pl.control_bytes, stream);
+    return err == cudaSuccess ? SABLOCK_OK : note_cuda_error(err, "clearing the control words");
 }
 
 // ------------------------------------------------------------------ stage launchers
@@ -349,10 +360,11 @@ sablock_status_t run_score(const Plan& pl, const sablock_params_t* p, const void
             fa.s_out = s; fa.e_out = e; fa.status = status;
             Geo geo = g;
             void* args[] = {&tmQ, &tmK, &geo, &fa};
-            if (cudaLaunchCooperativeKernel((const void*)score_fused_tc, dim3(groups * cpp), dim3(kFuThreads), args,
-                                            kFuSmemBytes, stream) != cudaSuccess) {
+            const cudaError_t err = cudaLaunchCooperativeKernel((const void*)score_fused_tc, dim3(groups * cpp), dim3(kFuThreads),
+                                                                args, kFuSmemBytes, stream);
+            if (err != cudaSuccess) {
                 cudaGetLastError();
-                return SABLOCK_ERR_CUDA;
+                return note_cuda_error(err, "cooperative launch of the score kernel");
             }
             ++t_launches;
             prof_mark(1, stream);
@@ -465,10 +477,11 @@ sablock_status_t run_select(const Plan& pl, const sablock_params_t* p, const flo
             Geo geo = g;
             const float* sr = s_ref;
             void* args[] = {&geo, &sr, &thr, &cut, &tsc, &status};
-            if (cudaLaunchCooperativeKernel((const void*)topb_kernel, dim3(ctas, pl.n_prob), dim3(kTopThreads), args, 0, stream) !=
-                cudaSuccess) {
+            const cudaError_t err =
+                cudaLaunchCooperativeKernel((const void*)topb_kernel, dim3(ctas, pl.n_prob), dim3(kTopThreads), args, 0, stream);
+            if (err != cudaSuccess) {
                 cudaGetLastError();
-                return SABLOCK_ERR_CUDA;
+                return note_cuda_error(err, "cooperative launch of the top-B kernel");
             }
             ++t_launches;
         } else {
@@ -540,6 +553,8 @@ void sablock_params_default(sablock_params_t* p)
     p->budget_includes_window = 1;
     p->score_impl = SABLOCK_SCORE_AUTO;
 }
+
+const char* sablock_last_cuda_error(void) { return t_cuda_error; }
 
 const char* sablock_status_string(sablock_status_t st)
 {
