@@ -62,6 +62,16 @@ constexpr int kFuSmemBytes = 1024 + (kFuQBufs + kFuStages) * kFuTileBytes;
 // settle half a step apart and one computes while the other waits, loads and fetches its next
 // step, instead of both doing so at the same time.
 constexpr int kReleaseAt = SABLOCK_RELEASE_AT;
+#ifndef SABLOCK_XU_TURNS
+#define SABLOCK_XU_TURNS 1
+#endif
+// The two epilogue sets take turns at the exponentials.  The special-function unit is the busiest
+// unit of the kernel; two sets that share it freely end up in lockstep, both computing and then
+// both going through the latencies between two steps (step record, accumulator barrier,
+// tensor-memory loads) with the unit idle.  With turns, set s starts the exponentials of its k-th
+// step only when the other set is halfway through those of its own preceding step, which keeps
+// the sets half a step apart: while one goes through the latencies the other has the unit.
+constexpr bool kXuTurns = SABLOCK_XU_TURNS != 0;
 
 struct FusedArgs {
     int cpp;                 // CTAs per group (one group works on one problem at a time)
@@ -84,7 +94,7 @@ struct FusedArgs {
 // merged; 5: merges of all CTAs in, log-sum-exps fetched).
 #ifdef SABLOCK_TRACE
 constexpr int kTraceOps = 600;
-__device__ long long g_trace[4][6][kTraceOps][4];   // [traced CTA][role][step][event]
+__device__ long long g_trace[4][6][kTraceOps][8];   // [traced CTA][role][step][event]
 #define FU_TRACE(role, n, ev)                                                                 \
     do {                                                                                      \
         if (tslot >= 0 && (n) < kTraceOps) g_trace[tslot][role][n][ev] = clock64();           \
@@ -103,6 +113,7 @@ struct FuBarriers {
     uint64_t pbar[2][4];     // the two warps of one set that share a tensor-memory lane quarter
     uint64_t pub_full[2];    // row sums of a phase are in shared memory (all epilogue threads)
     uint64_t lse_full[kFuLseSlots];
+    uint64_t xu[2];          // turn of epilogue set s at the exponentials
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -477,6 +488,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             for (int q = 0; q < 4; ++q) mbar_init(smem_u32(&sh.pbar[i][q]), 64);
         }
         for (int i = 0; i < kFuLseSlots; ++i) mbar_init(smem_u32(&sh.lse_full[i]), 1);
+        for (int i = 0; i < 2; ++i) mbar_init(smem_u32(&sh.xu[i]), kFuEpiWarps * 16);
         sh.abort_flag = 0;
         sched.count = 0;
         sched.final_ = 0;
@@ -792,7 +804,10 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         chunk_mask(r0, tok0, lim);
                         chunk_mask(r1, tok0 + 32, lim);
                     }
+                    if (kXuTurns && !FU_WAIT(9, mbar_wait(smem_u32(&sh.xu[set]), (uint32_t)((n_mine & 1) ^ (set ^ 1)), abort_flag))) break;
+                    if (first_thread) FU_TRACE(2 + set, n_mine, 6);
                     rs.add(r0, c2);
+                    if (kXuTurns) mbar_arrive(smem_u32(&sh.xu[set ^ 1]));
                     if (kReleaseAt == 1) mbar_arrive(smem_u32(&sh.tempty[set]));
                     rs.add(r1, c2);
                     if (kReleaseAt == 2) mbar_arrive(smem_u32(&sh.tempty[set]));
@@ -840,12 +855,16 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     tc_fence_before();
                     if (kReleaseAt == 0) mbar_arrive(smem_u32(&sh.tempty[set]));
                     if (first_thread) FU_TRACE(2 + set, n_mine, 2);
+                    if (kXuTurns && !FU_WAIT(9, mbar_wait(smem_u32(&sh.xu[set]), (uint32_t)((n_mine & 1) ^ (set ^ 1)), abort_flag))) break;
+                    if (first_thread) FU_TRACE(2 + set, n_mine, 6);
                     accumulate_head16(accw, v0, lj, c2);
                     accumulate_head16(accw, v1, lj + 32, c2);
+                    if (kXuTurns) mbar_arrive(smem_u32(&sh.xu[set ^ 1]));
                     if (kReleaseAt == 1) mbar_arrive(smem_u32(&sh.tempty[set]));
                     accumulate_head16(accw, v2, lj + 64, c2);
                     accumulate_head16(accw, v3, lj + 96, c2);
                     if (kReleaseAt == 2) mbar_arrive(smem_u32(&sh.tempty[set]));
+                    if (first_thread) FU_TRACE(2 + set, n_mine, 7);
                     // \bar A of this token tile, summed over the KV heads seen so far
                     const uint32_t abar_addr = lane_addr + (uint32_t)(kFuAbarCol0 + ((flags >> kStepKShift) & 7) * 32 + half * 16);
                     if (!(flags & kStepHead0)) {
