@@ -62,6 +62,9 @@ constexpr int kFuSmemBytes = 1024 + (kFuQBufs + kFuStages) * kFuTileBytes;
 // settle half a step apart and one computes while the other waits, loads and fetches its next
 // step, instead of both doing so at the same time.
 constexpr int kReleaseAt = SABLOCK_RELEASE_AT;
+#ifndef SABLOCK_F32X2
+#define SABLOCK_F32X2 1
+#endif
 #ifndef SABLOCK_XU_TURNS
 #define SABLOCK_XU_TURNS 1
 #endif
@@ -95,9 +98,14 @@ struct FusedArgs {
 #ifdef SABLOCK_TRACE
 constexpr int kTraceOps = 600;
 __device__ long long g_trace[4][6][kTraceOps][8];   // [traced CTA][role][step][event]
+#ifdef SABLOCK_TRACE_MIN       // epilogue: only "accumulator released" and "step done", to keep the probes' own cost out
+#define FU_TRACE_KEEP(role, ev) ((role) < 2 || (role) > 3 || (ev) == 2 || (ev) == 3 || (ev) == SABLOCK_TRACE_MIN || (SABLOCK_TRACE_MIN == 67 && ((ev) == 6 || (ev) == 7)))
+#else
+#define FU_TRACE_KEEP(role, ev) true
+#endif
 #define FU_TRACE(role, n, ev)                                                                 \
     do {                                                                                      \
-        if (tslot >= 0 && (n) < kTraceOps) g_trace[tslot][role][n][ev] = clock64();           \
+        if (FU_TRACE_KEEP(role, ev) && tslot >= 0 && (n) < kTraceOps) g_trace[tslot][role][n][ev] = clock64(); \
     } while (0)
 #else
 #define FU_TRACE(role, n, ev) do { } while (0)
@@ -224,7 +232,8 @@ struct FuIter {
 // One tile step as the other roles see it: 16 bytes in the shared-memory ring.
 constexpr int kStepB = 1 << 0;          // sweep B (else sweep A)
 constexpr int kStepLastA = 1 << 1;      // last sweep A step of its phase for this CTA: row sums are due
-constexpr int kStepFirstB = 1 << 3;     // first sweep B step of its phase for this CTA: next log-sum-exp buffer
+constexpr int kStepPrevLastA = 1 << 2;  // (epilogue rings) the step before this one, taken by the other set, was a kStepLastA step
+constexpr int kStepLseWait = 1 << 3;    // (epilogue rings) first sweep B step of its phase for this set: wait for the log-sum-exps
 constexpr int kStepKShift = 4;          // bits 4-6: slot of the tile among the CTA's tiles
 constexpr int kStepHead0 = 1 << 7;      // first KV head of the layer (sweep B starts \bar A afresh)
 constexpr int kStepHeadLast = 1 << 8;   // last KV head of the layer (sweep B emits s and the entropy)
@@ -233,10 +242,18 @@ constexpr int kStepQPar = 1 << 11;      // parity of that buffer's load
 constexpr int kStepRelShift = 12;       // bits 12-14: before this step, query-block buffer i has seen its last product
 constexpr int kStepMask = 1 << 15;      // sweep A tile that reaches the causal boundary
 constexpr int kStepNewQ = 1 << 16;      // first step that uses this load of the query block
+constexpr int kStepLseShift = 17;       // (epilogue rings) bits 17-18: log-sum-exp buffer of the phase, bit 19: parity of its fill
+constexpr int kStepStop = 1 << 20;      // (epilogue rings) no further step for this set
+constexpr int kStepTagShift = 24;       // (epilogue rings) bits 24-31: which use of the ring slot this is (never 0)
 
 constexpr int kFuRing = 16;
+constexpr int kFuSetRing = 8;
 struct FuSched {
     int4 ring[kFuRing];      // {flags, first token of the tile, T of the sequence, row offset of the outputs}
+    // The steps of each epilogue set once more, in a ring of its own: a set reads only its own
+    // steps (what it must know about the other set's steps is folded into the flags), and a
+    // record says by its tag whether it has been posted, so one look at the slot is enough.
+    int4 sring[2][kFuSetRing];
     volatile int count;      // steps posted so far
     volatile int final_;     // the producer has posted its last step
     volatile int lse_fetched;   // log-sum-exp buffers filled so far (helper warp)
@@ -375,6 +392,36 @@ __device__ __forceinline__ bool sched_get(FuSched& sc, int idx, int4& out, volat
     return true;
 }
 
+// Posts the k-th step of an epilogue set: payload first, then the tagged flags word.
+__device__ __forceinline__ void sched_post_set(FuSched& sc, int set, int k, int4 step)
+{
+    const uint32_t dst = smem_u32(&sc.sring[set][k % kFuSetRing]);
+    const int tag = ((k / kFuSetRing) & 0x7f) + 1;
+    asm volatile("st.volatile.shared.s32 [%0], %1;" ::"r"(dst + 4), "r"(step.y) : "memory");
+    asm volatile("st.volatile.shared.v2.s32 [%0], {%1, %2};" ::"r"(dst + 8), "r"(step.z), "r"(step.w) : "memory");
+    asm volatile("st.volatile.shared.s32 [%0], %1;" ::"r"(dst), "r"(step.x | (tag << kStepTagShift)) : "memory");
+}
+// Reads the k-th step of an epilogue set, waiting (bounded) until it is posted.  The flags word is
+// read before the payload, so a matching tag means the payload is the one posted with it.
+__device__ __forceinline__ bool sched_get_set(FuSched& sc, int set, int k, int4& out, volatile int* abort_flag)
+{
+    const uint32_t src = smem_u32(&sc.sring[set][k % kFuSetRing]);
+    const int tag = ((k / kFuSetRing) & 0x7f) + 1;
+    long long t0 = 0;
+    int spins = 0;
+    while (true) {
+        int fl;
+        asm volatile("ld.volatile.shared.s32 %0, [%1];" : "=r"(fl) : "r"(src) : "memory");
+        asm volatile("ld.volatile.shared.v4.s32 {%0, %1, %2, %3}, [%4];" : "=r"(out.x), "=r"(out.y), "=r"(out.z), "=r"(out.w) : "r"(src) : "memory");
+        if (((unsigned)fl >> kStepTagShift) == (unsigned)tag) {
+            out.x = fl;
+            return true;
+        }
+        if (spins++ == 0) t0 = clock64();
+        if ((spins & 15) == 0 && (*abort_flag || clock64() - t0 > kWaitLimitCycles)) { *abort_flag = 1; return false; }
+    }
+}
+
 // First wait of the launch that gave up: (code, CTA, warp) goes to the word after the status word.
 __device__ __forceinline__ void note_giveup(int* status, int code)
 {
@@ -383,9 +430,56 @@ __device__ __forceinline__ void note_giveup(int* status, int code)
 #define FU_WAIT(code, expr) ((expr) ? true : (note_giveup(fa.status, code), false))
 
 // ---- arithmetic of the epilogue ---------------------------------------------------------------
+// Packed fp32 pairs (one instruction for two lanes of arithmetic: the epilogue is short of issue
+// slots, not of fp32 throughput).
+__device__ __forceinline__ uint64_t pack2(float lo, float hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ uint64_t pack2u(uint32_t lo, uint32_t hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b)
+{
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+
 // Sum of exp2(v * c2 - m) over 32 logits of one window row.
 __device__ __forceinline__ float chunk_expsum(const uint32_t (&r)[32], float c2, float m)
 {
+#if SABLOCK_F32X2
+    const uint64_t cc = pack2(c2, c2), mm = pack2(-m, -m);
+    uint64_t s0 = pack2(0.f, 0.f), s1 = s0;
+#pragma unroll
+    for (int i = 0; i < 32; i += 4) {
+        float a, b, c, d;
+        unpack2(fma2(pack2u(r[i + 0], r[i + 1]), cc, mm), a, b);
+        unpack2(fma2(pack2u(r[i + 2], r[i + 3]), cc, mm), c, d);
+        s0 = add2(s0, pack2(ex2_approx(a), ex2_approx(b)));
+        s1 = add2(s1, pack2(ex2_approx(c), ex2_approx(d)));
+    }
+    float a, b, c, d;
+    unpack2(s0, a, b);
+    unpack2(s1, c, d);
+    return (a + b) + (c + d);
+#else
     float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
     for (int i = 0; i < 32; i += 4) {
@@ -395,6 +489,7 @@ __device__ __forceinline__ float chunk_expsum(const uint32_t (&r)[32], float c2,
         s3 += ex2_approx(fmaf(__uint_as_float(r[i + 3]), c2, -m));
     }
     return (s0 + s1) + (s2 + s3);
+#endif
 }
 __device__ __forceinline__ float chunk_max(const uint32_t (&r)[32])
 {
@@ -447,6 +542,18 @@ struct RowSum {
 __device__ __forceinline__ void accumulate_head16(float (&accw)[16], const uint32_t (&r)[16], const float* lse, float c2)
 {
     const float4* l4 = reinterpret_cast<const float4*>(lse);
+#if SABLOCK_F32X2
+    const uint64_t cc = pack2(c2, c2);
+#pragma unroll
+    for (int i = 0; i < 16; i += 4) {
+        const float4 ls = l4[i >> 2];
+        float a, b, c, d;
+        unpack2(fma2(pack2u(r[i + 0], r[i + 1]), cc, pack2(-ls.x, -ls.y)), a, b);
+        unpack2(fma2(pack2u(r[i + 2], r[i + 3]), cc, pack2(-ls.z, -ls.w)), c, d);
+        unpack2(add2(pack2(accw[i + 0], accw[i + 1]), pack2(ex2_approx(a), ex2_approx(b))), accw[i + 0], accw[i + 1]);
+        unpack2(add2(pack2(accw[i + 2], accw[i + 3]), pack2(ex2_approx(c), ex2_approx(d))), accw[i + 2], accw[i + 3]);
+    }
+#else
 #pragma unroll
     for (int i = 0; i < 16; i += 4) {
         const float4 ls = l4[i >> 2];
@@ -455,6 +562,7 @@ __device__ __forceinline__ void accumulate_head16(float (&accw)[16], const uint3
         accw[i + 2] += ex2_approx(fmaf(__uint_as_float(r[i + 2]), c2, -ls.z));
         accw[i + 3] += ex2_approx(fmaf(__uint_as_float(r[i + 3]), c2, -ls.w));
     }
+#endif
 }
 
 __global__ void __launch_bounds__(kFuThreads, 1)
@@ -491,6 +599,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         for (int i = 0; i < 2; ++i) mbar_init(smem_u32(&sh.xu[i]), kFuEpiWarps * 16);
         sh.abort_flag = 0;
         sched.count = 0;
+        for (int i = 0; i < 2 * kFuSetRing; ++i) (&sched.sring[0][0])[i] = make_int4(0, 0, 0, 0);
         sched.final_ = 0;
         sched.lse_fetched = 0;
         sched.pub_done = 0;
@@ -531,7 +640,8 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             }
             unsigned fq_par = 0;                               // the same parities as the work list sees them
             int q_phase = -1, pending_rel = 0, b_idx = -1, b_counted = -1, n_steps = 0;
-            bool ok = true;
+            int sb0 = -1, sb1 = -1;                            // last sweep B phase in which set 0 / set 1 had a step
+            bool ok = true, prev_last_a = false;
             while (ok) {
                 // ---- next step of the work list
                 if (it.b_pending() && b_counted != it.b_ph) {  // sweep B entered a phase: it needs the helper's next fetch
@@ -561,13 +671,27 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     }
                 } else {
                     flags |= kStepB;
-                    if (op.k == 0) flags |= kStepFirstB;
                     if (ph.j == 0) flags |= kStepHead0;
                     if (ph.j == g.Hkv - 1) flags |= kStepHeadLast;
                 }
                 if (ph.qpar) flags |= kStepQPar;
                 const int tok0 = op.tile * kTcTile;
-                sched_post(sched, n_steps, make_int4(flags, tok0, ph.Tn, ph.layer * g.total_tokens + ph.tok_base));
+                const int4 rec = make_int4(flags, tok0, ph.Tn, ph.layer * g.total_tokens + ph.tok_base);
+                sched_post(sched, n_steps, rec);
+                {
+                    const int eset = n_steps & 1;
+                    int ef = flags & ~(7 << kStepRelShift);
+                    if (prev_last_a) ef |= kStepPrevLastA;
+                    if (is_b) {
+                        ef |= ((b_idx % kFuLseSlots) | (((b_idx / kFuLseSlots) & 1) << 2)) << kStepLseShift;
+                        if ((eset ? sb1 : sb0) != b_idx) {
+                            if (eset) sb1 = b_idx; else sb0 = b_idx;
+                            ef |= kStepLseWait;
+                        }
+                    }
+                    sched_post_set(sched, eset, n_steps >> 1, make_int4(ef, rec.y, rec.z, rec.w));
+                    prev_last_a = !is_b && op.last;
+                }
                 FU_TRACE(0, n_steps, 3);
                 // ---- query blocks: this step's must be on its way (blocking); the next phase's is
                 // started if its buffer is free (probe only)
@@ -613,6 +737,13 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 ++n_steps;
             }
             sched.final_ = 1;
+            // the end of each epilogue set's list (also after a wait that gave up: the sets then
+            // leave through the abort flag)
+            for (int es = 0; es < 2; ++es) {
+                const int k = (n_steps + 1 - es) >> 1;         // steps set es has had
+                const bool other_was_last = prev_last_a && ((n_steps - 1) & 1) != es;
+                sched_post_set(sched, es, k, make_int4(kStepStop | (other_was_last ? kStepPrevLastA : 0), 0, 0, 0));
+            }
         }
     } else if (warp == 1 || warp == kFuMmaWarp2) {
         // ------------------------------------------------------------------ MMA issuers
@@ -779,14 +910,33 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         const float inv_H = 1.f / (float)g.H;
         RowSum rs;                                     // sweep A state of (window row, set, half)
         rs.reset();
-        int n = 0, n_mine = 0, n_lse = -1, lse_waited = -1, n_pub = 0, n_psync = 0, n_fin = 0;
+        int n_mine = 0, n_pub = 0, n_psync = 0, n_fin = 0;
+        // Hands this thread's row sum of a phase to the helper warp (no waiting unless the helper is
+        // two phases behind).
+        auto publish = [&]() -> bool {
+            const int buf = n_pub & 1;
+            if (n_pub >= 2 && sched.pub_done < n_pub - 1) {
+                const long long t0 = clock64();
+                while (sched.pub_done < n_pub - 1) {
+                    if (*abort_flag || clock64() - t0 > kWaitLimitCycles) { note_giveup(fa.status, 21); *abort_flag = 1; break; }
+                }
+                if (*abort_flag) return false;
+            }
+            pub_s[buf][set * 2 + half][row] = make_float2(rs.m, rs.l);
+            mbar_arrive(smem_u32(&sh.pub_full[buf]));
+            ++n_pub;
+            rs.reset();
+            return true;
+        };
         int4 e;
-        while (sched_get(sched, n, e, abort_flag)) {
+        while (sched_get_set(sched, set, n_mine, e, abort_flag)) {
             const int flags = e.x;
-            const bool mine = (n & 1) == set;
-            ++n;
+            if (first_thread) FU_TRACE(2 + set, n_mine, 5);
+            // the other set took the last sweep A step of a phase: this thread's row sums are due too
+            if ((flags & kStepPrevLastA) && !publish()) break;
+            if (flags & kStepStop) break;
             if (!(flags & kStepB)) {
-                if (mine) {
+                {
                     if (first_thread) FU_TRACE(2 + set, n_mine, 0);
                     if (!FU_WAIT(7, mbar_wait(smem_u32(&sh.tfull[set]), (uint32_t)(n_mine & 1), abort_flag))) break;
                     if (first_thread) FU_TRACE(2 + set, n_mine, 1);
@@ -814,35 +964,19 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     if (first_thread) FU_TRACE(2 + set, n_mine, 3);
                     ++n_mine;
                 }
-                if (flags & kStepLastA) {
-                    // Hand this thread's row sum of the phase to the helper warp (no waiting unless the
-                    // helper is two phases behind).
-                    const int buf = n_pub & 1;
-                    if (n_pub >= 2 && sched.pub_done < n_pub - 1) {
-                        const long long t0 = clock64();
-                        while (sched.pub_done < n_pub - 1) {
-                            if (*abort_flag || clock64() - t0 > kWaitLimitCycles) { note_giveup(fa.status, 21); *abort_flag = 1; break; }
-                        }
-                        if (*abort_flag) break;
-                    }
-                    pub_s[buf][set * 2 + half][row] = make_float2(rs.m, rs.l);
-                    mbar_arrive(smem_u32(&sh.pub_full[buf]));
-                    ++n_pub;
-                    rs.reset();
-                }
+                if ((flags & kStepLastA) && !publish()) break;
             } else {
-                if (flags & kStepFirstB) ++n_lse;                  // n_lse-th phase in which this CTA runs sweep B
-                if (mine) {
-                    if (n_lse != lse_waited) {                     // log-sum-exps of this phase (fetched by warp 18)
-                        lse_waited = n_lse;
-                        if (!FU_WAIT(8, mbar_wait(smem_u32(&sh.lse_full[n_lse % kFuLseSlots]), (uint32_t)((n_lse / kFuLseSlots) & 1), abort_flag)))
+                {
+                    const int lse_slot = (flags >> kStepLseShift) & 3;
+                    if (flags & kStepLseWait) {                    // log-sum-exps of this phase (fetched by warp 18)
+                        if (!FU_WAIT(8, mbar_wait(smem_u32(&sh.lse_full[lse_slot]), (uint32_t)((flags >> (kStepLseShift + 2)) & 1), abort_flag)))
                             break;
                     }
                     if (first_thread) FU_TRACE(2 + set, n_mine, 0);
                     if (!FU_WAIT(7, mbar_wait(smem_u32(&sh.tfull[set]), (uint32_t)(n_mine & 1), abort_flag))) break;
                     if (first_thread) FU_TRACE(2 + set, n_mine, 1);
                     tc_fence_after();
-                    const float* lj = lse_s[n_lse % kFuLseSlots] + half * 16;
+                    const float* lj = lse_s[lse_slot] + half * 16;
                     float accw[16];
 #pragma unroll
                     for (int i = 0; i < 16; ++i) accw[i] = 0.f;
