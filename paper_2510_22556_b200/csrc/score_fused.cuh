@@ -65,6 +65,10 @@ constexpr int kReleaseAt = SABLOCK_RELEASE_AT;
 #ifndef SABLOCK_F32X2
 #define SABLOCK_F32X2 1
 #endif
+#ifndef SABLOCK_AHEAD
+#define SABLOCK_AHEAD 1
+#endif
+constexpr bool kAhead = SABLOCK_AHEAD != 0;
 #ifndef SABLOCK_XU_TURNS
 #define SABLOCK_XU_TURNS 1
 #endif
@@ -107,8 +111,13 @@ __device__ long long g_trace[4][6][kTraceOps][8];   // [traced CTA][role][step][
     do {                                                                                      \
         if (FU_TRACE_KEEP(role, ev) && tslot >= 0 && (n) < kTraceOps) g_trace[tslot][role][n][ev] = clock64(); \
     } while (0)
+#define FU_TRACE_VAL(role, n, ev, val)                                                        \
+    do {                                                                                      \
+        if (tslot >= 0 && (n) < kTraceOps) g_trace[tslot][role][n][ev] = (val);               \
+    } while (0)
 #else
 #define FU_TRACE(role, n, ev) do { } while (0)
+#define FU_TRACE_VAL(role, n, ev, val) do { } while (0)
 #endif
 
 struct FuBarriers {
@@ -340,6 +349,31 @@ __device__ __forceinline__ void tmem_st_wait()
     asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
 
+// 2^d for an integer d <= 0, built from the exponent field (d below -126 gives 2^-126: the
+// product with any row sum is then far below one unit of the result).
+__device__ __forceinline__ float pow2_nonpos(int d)
+{
+    return __int_as_float((127 + max(d, -126)) << 23);
+}
+__device__ __forceinline__ int redux_max_s32(int v)
+{
+    int r;
+    asm volatile("redux.sync.max.s32 %0, %1, 0xffffffff;" : "=r"(r) : "r"(v));
+    return r;
+}
+__device__ __forceinline__ unsigned redux_max_u32(unsigned v)
+{
+    unsigned r;
+    asm volatile("redux.sync.max.u32 %0, %1, 0xffffffff;" : "=r"(r) : "r"(v));
+    return r;
+}
+__device__ __forceinline__ unsigned redux_add_u32(unsigned v)
+{
+    unsigned r;
+    asm volatile("redux.sync.add.u32 %0, %1, 0xffffffff;" : "=r"(r) : "r"(v));
+    return r;
+}
+
 // Bounded wait until *ctr >= target.  Gives up after about a second, or as soon as another
 // role of the CTA or another CTA has reported a failure.
 __device__ __forceinline__ bool wait_counter(const int* ctr, int target, volatile int* abort_flag, const int* status)
@@ -420,6 +454,25 @@ __device__ __forceinline__ bool sched_get_set(FuSched& sc, int set, int k, int4&
         if (spins++ == 0) t0 = clock64();
         if ((spins & 15) == 0 && (*abort_flag || clock64() - t0 > kWaitLimitCycles)) { *abort_flag = 1; return false; }
     }
+}
+
+// The flags word of the k-th step of an epilogue set as it stands (posted or not), and whether a
+// flags word read that way is the posted k-th step.
+__device__ __forceinline__ int sched_peek_flags(FuSched& sc, int set, int k)
+{
+    int fl;
+    asm volatile("ld.volatile.shared.s32 %0, [%1];" : "=r"(fl) : "r"(smem_u32(&sc.sring[set][k % kFuSetRing])) : "memory");
+    return fl;
+}
+__device__ __forceinline__ bool sched_flags_posted(int fl, int k)
+{
+    return ((unsigned)fl >> kStepTagShift) == (unsigned)(((k / kFuSetRing) & 0x7f) + 1);
+}
+// Payload of a step whose flags word has been seen posted.
+__device__ __forceinline__ void sched_payload(FuSched& sc, int set, int k, int4& out)
+{
+    asm volatile("ld.volatile.shared.v4.s32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(out.x), "=r"(out.y), "=r"(out.z), "=r"(out.w) : "r"(smem_u32(&sc.sring[set][k % kFuSetRing])) : "memory");
 }
 
 // First wait of the launch that gave up: (code, CTA, warp) goes to the word after the status word.
@@ -538,7 +591,7 @@ struct RowSum {
     }
 };
 
-// accw[i] += exp2(logit * c2 - lse) for 16 window positions of one query head.
+// accw[i] += exp2(logit * c2 - lse) for 16 window positions of one query head; `lse` holds -lse.
 __device__ __forceinline__ void accumulate_head16(float (&accw)[16], const uint32_t (&r)[16], const float* lse, float c2)
 {
     const float4* l4 = reinterpret_cast<const float4*>(lse);
@@ -548,8 +601,8 @@ __device__ __forceinline__ void accumulate_head16(float (&accw)[16], const uint3
     for (int i = 0; i < 16; i += 4) {
         const float4 ls = l4[i >> 2];
         float a, b, c, d;
-        unpack2(fma2(pack2u(r[i + 0], r[i + 1]), cc, pack2(-ls.x, -ls.y)), a, b);
-        unpack2(fma2(pack2u(r[i + 2], r[i + 3]), cc, pack2(-ls.z, -ls.w)), c, d);
+        unpack2(fma2(pack2u(r[i + 0], r[i + 1]), cc, pack2(ls.x, ls.y)), a, b);
+        unpack2(fma2(pack2u(r[i + 2], r[i + 3]), cc, pack2(ls.z, ls.w)), c, d);
         unpack2(add2(pack2(accw[i + 0], accw[i + 1]), pack2(ex2_approx(a), ex2_approx(b))), accw[i + 0], accw[i + 1]);
         unpack2(add2(pack2(accw[i + 2], accw[i + 3]), pack2(ex2_approx(c), ex2_approx(d))), accw[i + 2], accw[i + 3]);
     }
@@ -557,10 +610,10 @@ __device__ __forceinline__ void accumulate_head16(float (&accw)[16], const uint3
 #pragma unroll
     for (int i = 0; i < 16; i += 4) {
         const float4 ls = l4[i >> 2];
-        accw[i + 0] += ex2_approx(fmaf(__uint_as_float(r[i + 0]), c2, -ls.x));
-        accw[i + 1] += ex2_approx(fmaf(__uint_as_float(r[i + 1]), c2, -ls.y));
-        accw[i + 2] += ex2_approx(fmaf(__uint_as_float(r[i + 2]), c2, -ls.z));
-        accw[i + 3] += ex2_approx(fmaf(__uint_as_float(r[i + 3]), c2, -ls.w));
+        accw[i + 0] += ex2_approx(fmaf(__uint_as_float(r[i + 0]), c2, ls.x));
+        accw[i + 1] += ex2_approx(fmaf(__uint_as_float(r[i + 1]), c2, ls.y));
+        accw[i + 2] += ex2_approx(fmaf(__uint_as_float(r[i + 2]), c2, ls.z));
+        accw[i + 3] += ex2_approx(fmaf(__uint_as_float(r[i + 3]), c2, ls.w));
     }
 #endif
 }
@@ -572,7 +625,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     extern __shared__ uint8_t dyn_smem[];
     __shared__ FuBarriers sh;
     __shared__ __align__(16) FuSched sched;
-    __shared__ __align__(16) float lse_s[kFuLseSlots][128];      // log2-sum-exp2 of the window rows of a phase
+    __shared__ __align__(16) float lse_s[kFuLseSlots][128];      // minus the log2-sum-exp2 of the window rows of a phase
     __shared__ float2 pub_s[2][4][128];                          // [phase parity][set * 2 + half][window row]
     __shared__ float xch[2][2][2][2][128];                       // [set][use parity][tot | ent][half][token]
     const uint32_t base = (smem_u32(dyn_smem) + 1023u) & ~1023u;
@@ -769,6 +822,8 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         if (!FU_WAIT(3, mbar_wait(smem_u32(&sh.qfull[b]), (flags & kStepQPar) ? 1u : 0u, abort_flag))) break;
                     }
                     if (!FU_WAIT(4, mbar_wait(smem_u32(&sh.tempty[acc]), (uint32_t)((n_mine & 1) ^ 1), abort_flag))) break;
+                    FU_TRACE(1, n, 4);
+                    FU_TRACE_VAL(1, n, 5, flags);
                     if (!FU_WAIT(5, mbar_wait(smem_u32(&sh.full[st]), (uint32_t)par, abort_flag))) break;
                     FU_TRACE(1, n, 1);
                     tc_fence_after();
@@ -814,22 +869,24 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 if (!FU_WAIT(6, mbar_wait(smem_u32(&sh.pub_full[buf]), (uint32_t)((n_pub >> 1) & 1), abort_flag))) break;
                 if (lane == 0) FU_TRACE(4, phase, 0);
                 float2* dst = fa.part + (((size_t)group * kFuPartSlots + (phase % kFuPartSlots)) * fa.cpp + rank) * R;
+                // all partial sums of this lane's four rows first (the loads overlap), then the merges;
+                // the reference exponents are integers, so the rescaling is exact
+                float2 pv[4][4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+#pragma unroll
+                    for (int x = 0; x < 4; ++x) pv[u][x] = pub_s[buf][x][lane + 32 * u];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
-                    const int row = lane + 32 * u;
                     float m = -INFINITY;
 #pragma unroll
-                    for (int x = 0; x < 4; ++x) {
-                        const float2 v = pub_s[buf][x][row];
-                        if (v.y > 0.f) m = fmaxf(m, v.x);
-                    }
+                    for (int x = 0; x < 4; ++x)
+                        if (pv[u][x].y > 0.f) m = fmaxf(m, pv[u][x].x);
                     float l = 0.f;
 #pragma unroll
-                    for (int x = 0; x < 4; ++x) {
-                        const float2 v = pub_s[buf][x][row];
-                        if (v.y > 0.f) l += v.y * exp2f(v.x - m);     // exponents are integers: exact scaling
-                    }
-                    dst[row] = make_float2(l > 0.f ? m : 0.f, l);
+                    for (int x = 0; x < 4; ++x)
+                        if (pv[u][x].y > 0.f) l += pv[u][x].y * pow2_nonpos((int)(pv[u][x].x - m));
+                    dst[lane + 32 * u] = make_float2(l > 0.f ? m : 0.f, l);
                 }
                 __threadfence();
                 __syncwarp();
@@ -856,17 +913,27 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         const int i = lane + 32 * u;
                         v[u] = i < n_src ? __ldcg(pp + (size_t)i * R + row) : make_float2(0.f, 0.f);
                     }
-                    float m = -INFINITY;
+                    // Reference exponents are integer-valued: their maximum over the warp is an integer
+                    // reduction.  The sum over the warp is taken in fixed point relative to the
+                    // largest lane sum (26 bits each, 31 in all), so that it does not depend on an
+                    // order and needs one reduction instead of five exchanges.
+                    int mi = INT_MIN;
 #pragma unroll
                     for (int u = 0; u < kPer; ++u)
-                        if (v[u].y > 0.f) m = fmaxf(m, v[u].x);
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+                        if (v[u].y > 0.f) mi = max(mi, (int)v[u].x);
+                    mi = redux_max_s32(mi);
+                    const float m = (float)mi;
                     float l = 0.f;
 #pragma unroll
                     for (int u = 0; u < kPer; ++u)
-                        if (v[u].y > 0.f) l += v[u].y * exp2f(v[u].x - m);
-                    l = warp_sum(l);
+                        if (v[u].y > 0.f) l += v[u].y * pow2_nonpos((int)v[u].x - mi);
+                    const unsigned lmax = redux_max_u32(__float_as_uint(l));      // l >= 0: bit pattern orders like the value
+                    if (lmax != 0u) {
+                        const int ex = min(max((int)(lmax >> 23) - 127, -100), 100);   // 2^ex <= largest lane sum < 2^(ex + 1)
+                        const float up = __int_as_float((127 + 25 - ex) << 23), down = __int_as_float((127 - 25 + ex) << 23);
+                        const unsigned q = (unsigned)(l * up + 0.5f);                 // < 2^26
+                        l = (float)redux_add_u32(q) * down;
+                    }
                     if (lane == 0) fa.lse2[(size_t)prob * g.H * g.window + j * R + row] = m + log2f(l);
                 }
                 __syncwarp();
@@ -885,7 +952,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 const int slot = n_fetch % kFuLseSlots;
                 const float* src = fa.lse2 + (size_t)prob * g.H * g.window + j * R;
 #pragma unroll
-                for (int u = 0; u < 4; ++u) lse_s[slot][lane + 32 * u] = __ldcg(src + lane + 32 * u);
+                for (int u = 0; u < 4; ++u) lse_s[slot][lane + 32 * u] = -__ldcg(src + lane + 32 * u);   // negated: the epilogue adds it
                 __syncwarp();
                 ++n_fetch;
                 if (lane == 0) {
@@ -929,16 +996,29 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             return true;
         };
         int4 e;
-        while (sched_get_set(sched, set, n_mine, e, abort_flag)) {
+        // Read ahead during a step's exponentials, so that the latencies do not add up between two
+        // steps: the flags of the set's next step, and whether its accumulator is complete already.
+        int ahead_flags = 0;
+        bool ahead_tfull = false, have_payload = true;
+        while (true) {
+            if (kAhead && sched_flags_posted(ahead_flags, n_mine)) {
+                e.x = ahead_flags;
+                have_payload = false;
+            } else {
+                if (!sched_get_set(sched, set, n_mine, e, abort_flag)) break;
+                have_payload = true;
+                ahead_tfull = false;
+            }
             const int flags = e.x;
             if (first_thread) FU_TRACE(2 + set, n_mine, 5);
+            if (first_thread) FU_TRACE_VAL(2 + set, n_mine, 4, flags);
             // the other set took the last sweep A step of a phase: this thread's row sums are due too
             if ((flags & kStepPrevLastA) && !publish()) break;
             if (flags & kStepStop) break;
             if (!(flags & kStepB)) {
                 {
                     if (first_thread) FU_TRACE(2 + set, n_mine, 0);
-                    if (!FU_WAIT(7, mbar_wait(smem_u32(&sh.tfull[set]), (uint32_t)(n_mine & 1), abort_flag))) break;
+                    if (!ahead_tfull && !FU_WAIT(7, mbar_wait(smem_u32(&sh.tfull[set]), (uint32_t)(n_mine & 1), abort_flag))) break;
                     if (first_thread) FU_TRACE(2 + set, n_mine, 1);
                     tc_fence_after();
                     uint32_t r0[32], r1[32];
@@ -949,6 +1029,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     if (kReleaseAt == 0) mbar_arrive(smem_u32(&sh.tempty[set]));   // logits are in registers
                     if (first_thread) FU_TRACE(2 + set, n_mine, 2);
                     if (flags & kStepMask) {
+                        if (!have_payload) sched_payload(sched, set, n_mine, e);
                         const int tok0 = e.y + half * 64;
                         const int lim = e.z + (row & 31);          // causal: key index <= T + w (Eq. 2)
                         chunk_mask(r0, tok0, lim);
@@ -959,8 +1040,11 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     rs.add(r0, c2);
                     if (kXuTurns) mbar_arrive(smem_u32(&sh.xu[set ^ 1]));
                     if (kReleaseAt == 1) mbar_arrive(smem_u32(&sh.tempty[set]));
+                    if (kAhead) ahead_flags = sched_peek_flags(sched, set, n_mine + 1);
                     rs.add(r1, c2);
+                    if (kAhead) ahead_tfull = mbar_test_wait(smem_u32(&sh.tfull[set]), (uint32_t)((n_mine + 1) & 1));
                     if (kReleaseAt == 2) mbar_arrive(smem_u32(&sh.tempty[set]));
+                    if (first_thread) FU_TRACE(2 + set, n_mine, 7);
                     if (first_thread) FU_TRACE(2 + set, n_mine, 3);
                     ++n_mine;
                 }
@@ -973,7 +1057,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                             break;
                     }
                     if (first_thread) FU_TRACE(2 + set, n_mine, 0);
-                    if (!FU_WAIT(7, mbar_wait(smem_u32(&sh.tfull[set]), (uint32_t)(n_mine & 1), abort_flag))) break;
+                    if (!ahead_tfull && !FU_WAIT(7, mbar_wait(smem_u32(&sh.tfull[set]), (uint32_t)(n_mine & 1), abort_flag))) break;
                     if (first_thread) FU_TRACE(2 + set, n_mine, 1);
                     tc_fence_after();
                     const float* lj = lse_s[lse_slot] + half * 16;
@@ -995,8 +1079,10 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     accumulate_head16(accw, v1, lj + 32, c2);
                     if (kXuTurns) mbar_arrive(smem_u32(&sh.xu[set ^ 1]));
                     if (kReleaseAt == 1) mbar_arrive(smem_u32(&sh.tempty[set]));
+                    if (kAhead) ahead_flags = sched_peek_flags(sched, set, n_mine + 1);
                     accumulate_head16(accw, v2, lj + 64, c2);
                     accumulate_head16(accw, v3, lj + 96, c2);
+                    if (kAhead) ahead_tfull = mbar_test_wait(smem_u32(&sh.tfull[set]), (uint32_t)((n_mine + 1) & 1));
                     if (kReleaseAt == 2) mbar_arrive(smem_u32(&sh.tempty[set]));
                     if (first_thread) FU_TRACE(2 + set, n_mine, 7);
                     // \bar A of this token tile, summed over the KV heads seen so far
@@ -1033,6 +1119,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         }
                         xch[set][par][1][half][row] = ent_h;
                         if (!FU_WAIT(20, group_sync(&sh.pbar[set][q4], n_psync, abort_flag))) break;
+                        if (!have_payload) sched_payload(sched, set, n_mine, e);
                         const int t = e.y + row;
                         if (half == 0 && t < e.z) {
                             fa.s_out[(size_t)e.w + t] = tot * inv_H;
