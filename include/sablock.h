@@ -88,7 +88,10 @@ void sablock_params_default(sablock_params_t *p);
 const char *sablock_status_string(sablock_status_t st);
 int sablock_version(void);
 /* Text of the most recent CUDA runtime error an entry point of this thread ran into (which call,
- * after how many kernel launches of that entry point, and the runtime's message); "" if none. */
+ * after how many kernel launches of that entry point, and the runtime's message); "" if none.
+ * With SABLOCK_DEBUG_SYNC=1 in the environment sablock_compress_layers waits for the stream after
+ * every stage, so that a device fault is reported here with the stage that raised it (diagnostic
+ * aid; it serialises host and device). */
 const char *sablock_last_cuda_error(void);
 size_t sablock_params_sizeof(void);   /* sizeof(sablock_params_t) as the library was built */
 

@@ -112,6 +112,17 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
+// Optional counters of the polls of the bounded waits (compiled in with -DSABLOCK_TRACE).
+#ifdef SABLOCK_TRACE
+__device__ unsigned long long g_spin[8];
+#define SPIN_COUNT(i, n)                                                                      \
+    do {                                                                                      \
+        if ((threadIdx.x & 31) == 0 && (n) > 0) atomicAdd(&g_spin[i], (unsigned long long)(n)); \
+    } while (0)
+#else
+#define SPIN_COUNT(i, n) do { } while (0)
+#endif
+
 // Bounded wait: polls the barrier; gives up after `limit` clock cycles or as soon as another
 // role of the CTA has raised *abort.  Returns false on give-up (and raises *abort itself).
 constexpr long long kWaitLimitCycles = 2000000000LL;   // about one second
@@ -121,7 +132,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     long long t0 = clock64();
     int spins = 0;
     while (true) {
-        if (mbar_try_wait(bar, parity)) return true;
+        if (mbar_try_wait(bar, parity)) {
+            SPIN_COUNT(0, spins + 1);
+            SPIN_COUNT(5, 1);
+            return true;
+        }
 #ifdef SABLOCK_WAIT_SLEEP_NS
         __nanosleep(SABLOCK_WAIT_SLEEP_NS);
 #endif

@@ -3,6 +3,7 @@
 // the kernels of stages.cuh / score_simt.cuh / score_tc.cuh; there is no host fallback.
 #include <math.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include "common.cuh"
@@ -238,6 +239,16 @@ sablock_status_t check_launch()
     return err == cudaSuccess ? SABLOCK_OK : note_cuda_error(err, "kernel launch");
 }
 #define SAB_TRY(expr) do { sablock_status_t _s = (expr); if (_s != SABLOCK_OK) return _s; } while (0)
+
+// Diagnostic aid: with SABLOCK_DEBUG_SYNC=1 in the environment the pipeline waits for the stream
+// after every stage, so that a device fault is reported with the stage that raised it.
+sablock_status_t debug_sync(const char* stage, cudaStream_t stream)
+{
+    static const bool on = [] { const char* e = getenv("SABLOCK_DEBUG_SYNC"); return e && e[0] == '1'; }();
+    if (!on) return SABLOCK_OK;
+    const cudaError_t err = cudaStreamSynchronize(stream);
+    return err == cudaSuccess ? SABLOCK_OK : note_cuda_error(err, stage);
+}
 
 sablock_status_t zero_control(const Plan& pl, void* ws, cudaStream_t stream)
 {
@@ -796,15 +807,20 @@ sablock_status_t sablock_compress_layers(const sablock_params_t* p, int n_layers
     float* s_raw = p->pool_kernel > 1 ? at<float>(ws, pl.o_s_raw) : s;
     SAB_TRY(run_segment(pl, p, token_ids, seg_id, seg_start, n_seg, ws, st));
     prof_mark(0, st);
+    SAB_TRY(debug_sync("stage segment", st));
     SAB_TRY(run_score(pl, p, q_win, k, s_raw, e, ws, st));
     prof_mark(3, st);
+    SAB_TRY(debug_sync("stage score", st));
     SAB_TRY(run_refine(pl, p, s_raw, s, e, seg_start, n_seg, sr, nullptr, 0, st));
     prof_mark(4, st);
+    SAB_TRY(debug_sync("stage refine", st));
     SAB_TRY(run_select(pl, p, sr, seg_start, n_seg, cands, out_idx, out_n_keep, nullptr, nullptr, 0, ws, st));
     prof_mark(7, st);
+    SAB_TRY(debug_sync("stage select", st));
     sablock_status_t rc = run_compact(pl.geo, pl.n_prob, p, k, v, out_idx, out_n_keep, 0, out_k, out_v, st);
     prof_mark(8, st);
     prof_end_call();
+    if (rc == SABLOCK_OK) rc = debug_sync("stage compact", st);
     return rc;
 }
 
