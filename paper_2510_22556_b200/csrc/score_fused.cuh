@@ -594,9 +594,7 @@ struct RowSum {
     }
 };
 
-// accw[i] (+)= exp2(logit * c2 - lse) for 16 window positions of one query head; `lse` holds -lse.
-// kFirst: the sums start with this head (no zero-filled accumulators to add to).
-template <bool kFirst = false>
+// accw[i] += exp2(logit * c2 - lse) for 16 window positions of one query head; `lse` holds -lse.
 __device__ __forceinline__ void accumulate_head16(float (&accw)[16], const uint32_t (&r)[16], const float* lse, float c2)
 {
     const float4* l4 = reinterpret_cast<const float4*>(lse);
@@ -608,24 +606,17 @@ __device__ __forceinline__ void accumulate_head16(float (&accw)[16], const uint3
         float a, b, c, d;
         unpack2(fma2(pack2u(r[i + 0], r[i + 1]), cc, pack2(ls.x, ls.y)), a, b);
         unpack2(fma2(pack2u(r[i + 2], r[i + 3]), cc, pack2(ls.z, ls.w)), c, d);
-        if (kFirst) {
-            accw[i + 0] = ex2_approx(a);
-            accw[i + 1] = ex2_approx(b);
-            accw[i + 2] = ex2_approx(c);
-            accw[i + 3] = ex2_approx(d);
-        } else {
-            unpack2(add2(pack2(accw[i + 0], accw[i + 1]), pack2(ex2_approx(a), ex2_approx(b))), accw[i + 0], accw[i + 1]);
-            unpack2(add2(pack2(accw[i + 2], accw[i + 3]), pack2(ex2_approx(c), ex2_approx(d))), accw[i + 2], accw[i + 3]);
-        }
+        unpack2(add2(pack2(accw[i + 0], accw[i + 1]), pack2(ex2_approx(a), ex2_approx(b))), accw[i + 0], accw[i + 1]);
+        unpack2(add2(pack2(accw[i + 2], accw[i + 3]), pack2(ex2_approx(c), ex2_approx(d))), accw[i + 2], accw[i + 3]);
     }
 #else
 #pragma unroll
     for (int i = 0; i < 16; i += 4) {
         const float4 ls = l4[i >> 2];
-        accw[i + 0] = (kFirst ? 0.f : accw[i + 0]) + ex2_approx(fmaf(__uint_as_float(r[i + 0]), c2, ls.x));
-        accw[i + 1] = (kFirst ? 0.f : accw[i + 1]) + ex2_approx(fmaf(__uint_as_float(r[i + 1]), c2, ls.y));
-        accw[i + 2] = (kFirst ? 0.f : accw[i + 2]) + ex2_approx(fmaf(__uint_as_float(r[i + 2]), c2, ls.z));
-        accw[i + 3] = (kFirst ? 0.f : accw[i + 3]) + ex2_approx(fmaf(__uint_as_float(r[i + 3]), c2, ls.w));
+        accw[i + 0] += ex2_approx(fmaf(__uint_as_float(r[i + 0]), c2, ls.x));
+        accw[i + 1] += ex2_approx(fmaf(__uint_as_float(r[i + 1]), c2, ls.y));
+        accw[i + 2] += ex2_approx(fmaf(__uint_as_float(r[i + 2]), c2, ls.z));
+        accw[i + 3] += ex2_approx(fmaf(__uint_as_float(r[i + 3]), c2, ls.w));
     }
 #endif
 }
@@ -1075,6 +1066,8 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     tc_fence_after();
                     const float* lj = lse_s[lse_slot] + half * 16;
                     float accw[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) accw[i] = 0.f;
                     uint32_t v0[16], v1[16], v2[16], v3[16];       // query head hl of the group, 16 window positions
                     tmem_ld16_issue(acc_addr + half * 16, v0);
                     tmem_ld16_issue(acc_addr + 32 + half * 16, v1);
@@ -1086,7 +1079,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     if (first_thread) FU_TRACE(2 + set, n_mine, 2);
                     if (kXuTurns && !FU_WAIT(9, mbar_wait(smem_u32(&sh.xu[set]), (uint32_t)((n_mine & 1) ^ (set ^ 1)), abort_flag))) break;
                     if (first_thread) FU_TRACE(2 + set, n_mine, 6);
-                    accumulate_head16<true>(accw, v0, lj, c2);
+                    accumulate_head16(accw, v0, lj, c2);
                     accumulate_head16(accw, v1, lj + 32, c2);
                     if (kXuTurns) mbar_arrive(smem_u32(&sh.xu[set ^ 1]));
                     if (kReleaseAt == 1) mbar_arrive(smem_u32(&sh.tempty[set]));
@@ -1102,8 +1095,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         tmem_ld16_issue(abar_addr, v0);
                         tmem_ld_wait();
 #pragma unroll
-                        for (int i = 0; i < 16; i += 2)
-                            unpack2(add2(pack2(accw[i], accw[i + 1]), pack2u(v0[i], v0[i + 1])), accw[i], accw[i + 1]);
+                        for (int i = 0; i < 16; ++i) accw[i] += __uint_as_float(v0[i]);
                     }
                     if (!(flags & kStepHeadLast)) {
                         tmem_st16(abar_addr, accw);
