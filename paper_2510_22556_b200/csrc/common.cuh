@@ -123,6 +123,25 @@ __device__ unsigned long long g_spin[8];
 #define SPIN_COUNT(i, n) do { } while (0)
 #endif
 
+// Non-blocking probes of two barriers whose latencies overlap (both tests are issued before
+// either result is used).
+__device__ __forceinline__ void mbar_test_wait2(uint32_t bar_a, uint32_t parity_a, uint32_t bar_b, uint32_t parity_b,
+                                                bool& ok_a, bool& ok_b)
+{
+    uint32_t a, b;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%2], %3;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 q, [%4], %5;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t"
+        "selp.u32 %1, 1, 0, q;\n\t}"
+        : "=r"(a), "=r"(b)
+        : "r"(bar_a), "r"(parity_a), "r"(bar_b), "r"(parity_b)
+        : "memory");
+    ok_a = a != 0;
+    ok_b = b != 0;
+}
+
 // Bounded wait: polls the barrier; gives up after `limit` clock cycles or as soon as another
 // role of the CTA has raised *abort.  Returns false on give-up (and raises *abort itself).
 constexpr long long kWaitLimitCycles = 2000000000LL;   // about one second

@@ -33,17 +33,30 @@
 
 namespace sab {
 
-constexpr int kFuThreads = 640;
+#ifndef SABLOCK_MMA_ISSUERS
+#define SABLOCK_MMA_ISSUERS 1
+#endif
+constexpr int kFuIssuers = SABLOCK_MMA_ISSUERS;   // threads that issue tcgen05.mma: 1, or 2 (one per accumulator)
+constexpr int kFuThreads = kFuIssuers == 2 ? 640 : 608;
 constexpr int kFuEpiWarp0 = 2;
 constexpr int kFuEpiWarps = 16;
 constexpr int kFuHelpWarp = 18;
 constexpr int kFuMmaWarp2 = 19;
-constexpr int kFuStages = 3;                 // K tile ring
-constexpr int kFuQBufs = 3;                  // query-block buffers: phases n - 1 (sweep B), n (sweep A), n + 1 (loading ahead)
+#ifndef SABLOCK_K_STAGES
+#define SABLOCK_K_STAGES 3
+#endif
+#ifndef SABLOCK_Q_BUFS
+#define SABLOCK_Q_BUFS 3
+#endif
+constexpr int kFuStages = SABLOCK_K_STAGES;   // K tile ring
+constexpr int kFuQBufs = SABLOCK_Q_BUFS;      // query-block buffers: phases n - 1 (sweep B), n (sweep A), n + 1 (loading ahead)
 constexpr int kFuMaxTilesPerCta = 7;         // \bar A slots in tensor memory: 7 x 32 columns
 constexpr int kFuAbarCol0 = 256;             // columns [0, 256): two logit accumulators
 constexpr int kFuTmemCols = 512;
-constexpr int kFuLead = 2;                   // sweep A runs at least this many tiles ahead of sweep B
+#ifndef SABLOCK_LEAD
+#define SABLOCK_LEAD 2
+#endif
+constexpr int kFuLead = SABLOCK_LEAD;                   // sweep A runs at least this many tiles ahead of sweep B
 #ifndef SABLOCK_RUN_AHEAD
 #define SABLOCK_RUN_AHEAD 0
 #endif
@@ -485,6 +498,30 @@ __device__ __forceinline__ void note_giveup(int* status, int code)
 }
 #define FU_WAIT(code, expr) ((expr) ? true : (note_giveup(fa.status, code), false))
 
+// One 128 x 128 x 128 product into accumulator `acc`: eight tcgen05.mma, unrolled, with the two
+// shared-memory descriptors built once (the k-steps only move the start-address field: 32 bytes
+// inside the 128-byte row, the second 64-column atom after the fourth step).  The issuing
+// thread shares its scheduler with four epilogue warps, so every instruction it saves counts.
+__device__ __forceinline__ void fu_issue_tile(uint32_t tmem, int acc, uint32_t a_base, uint32_t b_base)
+{
+    constexpr uint32_t idesc = umma_idesc_bf16(128, 128);
+    const uint64_t da = umma_desc_sw128(a_base), db = umma_desc_sw128(b_base);
+    const uint32_t d = tmem + (uint32_t)acc * 128u;
+#pragma unroll
+    for (int kk = 0; kk < 8; ++kk) {
+        constexpr uint32_t kAtom16 = kAtomBytes >> 4;
+        const uint32_t off16 = (uint32_t)(kk >> 2) * kAtom16 + (uint32_t)(kk & 3) * 2u;      // byte offset / 16
+        if (kk == 0)
+            asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, 0, 0;\n\t"
+                         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                         ::"r"(d), "l"(da + off16), "l"(db + off16), "r"(idesc) : "memory");
+        else
+            asm volatile("{\n\t.reg .pred p;\n\tsetp.eq.b32 p, 0, 0;\n\t"
+                         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                         ::"r"(d), "l"(da + off16), "l"(db + off16), "r"(idesc) : "memory");
+    }
+}
+
 // ---- arithmetic of the epilogue ---------------------------------------------------------------
 // Packed fp32 pairs (one instruction for two lanes of arithmetic: the epilogue is short of issue
 // slots, not of fp32 throughput).
@@ -643,7 +680,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         }
         for (int i = 0; i < kFuQBufs; ++i) {
             mbar_init(smem_u32(&sh.qfull[i]), 1);
-            mbar_init(smem_u32(&sh.qempty[i]), 2);
+            mbar_init(smem_u32(&sh.qempty[i]), kFuIssuers);
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&sh.tfull[i]), 1);
@@ -801,43 +838,65 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 sched_post_set(sched, es, k, make_int4(kStepStop | (other_was_last ? kStepPrevLastA : 0), 0, 0, 0));
             }
         }
-    } else if (warp == 1 || warp == kFuMmaWarp2) {
+    } else if (warp == 1 || (kFuIssuers == 2 && warp == kFuMmaWarp2)) {
         // ------------------------------------------------------------------ MMA issuers
         // One thread per accumulator: each issues the products of every other step, so that one can
         // wait for its barriers and read its next step while the other's products run.
         if (lane == 0) {
-            const int acc = warp == 1 ? 0 : 1;
-            int n = 0, n_mine = 0, q_gen[kFuQBufs] = {0, 0, 0}, q_seen[kFuQBufs] = {0, 0, 0};
-            int4 e;
-            while (sched_get(sched, n, e, abort_flag)) {
+            int n = 0, n_mine = 0, q_gen[kFuQBufs] = {}, q_seen[kFuQBufs] = {};
+            int4 e, e_next = make_int4(0, 0, 0, 0);
+            bool have_next = false;
+            while (true) {
+                if (have_next) e = e_next;
+                else if (!sched_get(sched, n, e, abort_flag)) break;
+                have_next = false;
                 const int flags = e.x;
 #pragma unroll
                 for (int i = 0; i < kFuQBufs; ++i)
                     if (flags & (1 << (kStepRelShift + i))) tc_commit(smem_u32(&sh.qempty[i]));
                 const int b = (flags >> kStepQBufShift) & 3;
-                if (flags & kStepNewQ) ++q_gen[b];
-                const bool mine = (n & 1) == acc;
+                if (kFuIssuers == 2 && (flags & kStepNewQ)) ++q_gen[b];
+                // with two issuers each takes the steps of one accumulator, with one it takes them all
+                const int acc = kFuIssuers == 2 ? (warp == 1 ? 0 : 1) : (n & 1);
+                const bool mine = kFuIssuers == 1 || (n & 1) == acc;
+                if (kFuIssuers == 1) n_mine = n >> 1;              // uses of this accumulator so far
                 const int st = n % kFuStages, par = (n / kFuStages) & 1;
                 if (mine) {
                     FU_TRACE(1, n, 0);
-                    if (q_seen[b] != q_gen[b]) {                   // this load of the query block
+                    // both barriers are probed before either result is looked at, so that their
+                    // latencies overlap; only a barrier that is not complete yet is waited for
+                    bool te_ok, k_ok;
+                    mbar_test_wait2(smem_u32(&sh.tempty[acc]), (uint32_t)((n_mine & 1) ^ 1), smem_u32(&sh.full[st]), (uint32_t)par,
+                                    te_ok, k_ok);
+                    // this load of the query block: its first product waits for it (a single issuer
+                    // takes every step, so that is the step flagged as the first user)
+                    bool new_q = (flags & kStepNewQ) != 0;
+                    if (kFuIssuers == 2) {
+                        new_q = q_seen[b] != q_gen[b];
                         q_seen[b] = q_gen[b];
-                        if (!FU_WAIT(3, mbar_wait(smem_u32(&sh.qfull[b]), (flags & kStepQPar) ? 1u : 0u, abort_flag))) break;
                     }
-                    if (!FU_WAIT(4, mbar_wait(smem_u32(&sh.tempty[acc]), (uint32_t)((n_mine & 1) ^ 1), abort_flag))) break;
+                    if (new_q && !FU_WAIT(3, mbar_wait(smem_u32(&sh.qfull[b]), (flags & kStepQPar) ? 1u : 0u, abort_flag))) break;
+                    if (!te_ok && !FU_WAIT(4, mbar_wait(smem_u32(&sh.tempty[acc]), (uint32_t)((n_mine & 1) ^ 1), abort_flag))) break;
                     FU_TRACE(1, n, 4);
                     FU_TRACE_VAL(1, n, 5, flags);
-                    if (!FU_WAIT(5, mbar_wait(smem_u32(&sh.full[st]), (uint32_t)par, abort_flag))) break;
+                    if (!k_ok && !FU_WAIT(5, mbar_wait(smem_u32(&sh.full[st]), (uint32_t)par, abort_flag))) break;
                     FU_TRACE(1, n, 1);
                     tc_fence_after();
+                    // the next step's record, if it is posted, comes in while the products are issued
+                    if (sched_count(sched) > n + 1) {
+                        const uint32_t src = smem_u32(&sched.ring[(n + 1) % kFuRing]);
+                        asm volatile("ld.volatile.shared.v4.s32 {%0, %1, %2, %3}, [%4];"
+                                     : "=r"(e_next.x), "=r"(e_next.y), "=r"(e_next.z), "=r"(e_next.w) : "r"(src) : "memory");
+                        have_next = true;
+                    }
                     const uint32_t kt = k_smem + st * kFuTileBytes, qt = q_smem + b * kFuTileBytes;
-                    if (flags & kStepB) tc_issue_tile(tmem, acc, kt, qt, 8);      // rows = tokens
-                    else                tc_issue_tile(tmem, acc, qt, kt, 8);      // rows = window rows
+                    const bool is_b = (flags & kStepB) != 0;
+                    fu_issue_tile(tmem, acc, is_b ? kt : qt, is_b ? qt : kt);      // rows = tokens (B) or window rows (A)
                     FU_TRACE(1, n, 2);
                     tc_commit(smem_u32(&sh.empty[st]));
                     tc_commit(smem_u32(&sh.tfull[acc]));
                     FU_TRACE(1, n, 3);
-                    ++n_mine;
+                    if (kFuIssuers == 2) ++n_mine;
                 }
                 ++n;
             }
