@@ -18,9 +18,9 @@
 // memory (32 columns per token tile) across the KV heads of a layer, so neither the H x W x T
 // attention tensor nor \bar A ever reaches shared or global memory.
 //
-// CTA = 20 warps.  Warp 0: one thread walks the work list, posts every tile step to a small ring
-// in shared memory and issues the TMA loads.  Warps 1 and 19: one MMA-issuing thread per
-// accumulator (warp 1 owns tensor memory).  Warps 2-17: epilogue, two sets of eight warps; set s
+// CTA = 19 warps.  Warp 0: one thread walks the work list, posts every tile step to a small ring
+// in shared memory and issues the TMA loads.  Warp 1: one thread issues every tcgen05.mma (the
+// warp owns tensor memory).  Warps 2-17: epilogue, two sets of eight warps; set s
 // takes the steps whose logits land in accumulator s, so one set computes while the other waits
 // and loads.  Inside a set two warps share each 32-lane quarter of tensor memory: in sweep A they
 // split the tile's 128 token columns, in sweep B the 32 window positions.  Warp 18: hand-over
@@ -33,15 +33,10 @@
 
 namespace sab {
 
-#ifndef SABLOCK_MMA_ISSUERS
-#define SABLOCK_MMA_ISSUERS 1
-#endif
-constexpr int kFuIssuers = SABLOCK_MMA_ISSUERS;   // threads that issue tcgen05.mma: 1, or 2 (one per accumulator)
-constexpr int kFuThreads = kFuIssuers == 2 ? 640 : 608;
+constexpr int kFuThreads = 608;
 constexpr int kFuEpiWarp0 = 2;
 constexpr int kFuEpiWarps = 16;
 constexpr int kFuHelpWarp = 18;
-constexpr int kFuMmaWarp2 = 19;
 #ifndef SABLOCK_K_STAGES
 #define SABLOCK_K_STAGES 3
 #endif
@@ -680,7 +675,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         }
         for (int i = 0; i < kFuQBufs; ++i) {
             mbar_init(smem_u32(&sh.qfull[i]), 1);
-            mbar_init(smem_u32(&sh.qempty[i]), kFuIssuers);
+            mbar_init(smem_u32(&sh.qempty[i]), 1);
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&sh.tfull[i]), 1);
@@ -838,12 +833,14 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 sched_post_set(sched, es, k, make_int4(kStepStop | (other_was_last ? kStepPrevLastA : 0), 0, 0, 0));
             }
         }
-    } else if (warp == 1 || (kFuIssuers == 2 && warp == kFuMmaWarp2)) {
-        // ------------------------------------------------------------------ MMA issuers
-        // One thread per accumulator: each issues the products of every other step, so that one can
-        // wait for its barriers and read its next step while the other's products run.
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        // One thread issues every product (the two accumulators alternate with the steps).  Issuing
+        // blocks for about as long as the tensor core needs for the tile, so everything else this
+        // thread does per step is kept short: no state in local memory, barrier probes whose
+        // latencies overlap, the next step's record fetched while the products are issued.
         if (lane == 0) {
-            int n = 0, n_mine = 0, q_gen[kFuQBufs] = {}, q_seen[kFuQBufs] = {};
+            int n = 0;
             int4 e, e_next = make_int4(0, 0, 0, 0);
             bool have_next = false;
             while (true) {
@@ -855,27 +852,17 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 for (int i = 0; i < kFuQBufs; ++i)
                     if (flags & (1 << (kStepRelShift + i))) tc_commit(smem_u32(&sh.qempty[i]));
                 const int b = (flags >> kStepQBufShift) & 3;
-                if (kFuIssuers == 2 && (flags & kStepNewQ)) ++q_gen[b];
-                // with two issuers each takes the steps of one accumulator, with one it takes them all
-                const int acc = kFuIssuers == 2 ? (warp == 1 ? 0 : 1) : (n & 1);
-                const bool mine = kFuIssuers == 1 || (n & 1) == acc;
-                if (kFuIssuers == 1) n_mine = n >> 1;              // uses of this accumulator so far
+                const int acc = n & 1, n_mine = n >> 1;            // accumulator of the step, its uses so far
                 const int st = n % kFuStages, par = (n / kFuStages) & 1;
-                if (mine) {
+                {
                     FU_TRACE(1, n, 0);
                     // both barriers are probed before either result is looked at, so that their
                     // latencies overlap; only a barrier that is not complete yet is waited for
                     bool te_ok, k_ok;
                     mbar_test_wait2(smem_u32(&sh.tempty[acc]), (uint32_t)((n_mine & 1) ^ 1), smem_u32(&sh.full[st]), (uint32_t)par,
                                     te_ok, k_ok);
-                    // this load of the query block: its first product waits for it (a single issuer
-                    // takes every step, so that is the step flagged as the first user)
-                    bool new_q = (flags & kStepNewQ) != 0;
-                    if (kFuIssuers == 2) {
-                        new_q = q_seen[b] != q_gen[b];
-                        q_seen[b] = q_gen[b];
-                    }
-                    if (new_q && !FU_WAIT(3, mbar_wait(smem_u32(&sh.qfull[b]), (flags & kStepQPar) ? 1u : 0u, abort_flag))) break;
+                    // the first product that uses a load of the query block waits for it
+                    if ((flags & kStepNewQ) && !FU_WAIT(3, mbar_wait(smem_u32(&sh.qfull[b]), (flags & kStepQPar) ? 1u : 0u, abort_flag))) break;
                     if (!te_ok && !FU_WAIT(4, mbar_wait(smem_u32(&sh.tempty[acc]), (uint32_t)((n_mine & 1) ^ 1), abort_flag))) break;
                     FU_TRACE(1, n, 4);
                     FU_TRACE_VAL(1, n, 5, flags);
@@ -896,7 +883,6 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     tc_commit(smem_u32(&sh.empty[st]));
                     tc_commit(smem_u32(&sh.tfull[acc]));
                     FU_TRACE(1, n, 3);
-                    if (kFuIssuers == 2) ++n_mine;
                 }
                 ++n;
             }
