@@ -493,28 +493,29 @@ __device__ __forceinline__ void note_giveup(int* status, int code)
 }
 #define FU_WAIT(code, expr) ((expr) ? true : (note_giveup(fa.status, code), false))
 
-// One 128 x 128 x 128 product into accumulator `acc`: eight tcgen05.mma, unrolled, with the two
-// shared-memory descriptors built once (the k-steps only move the start-address field: 32 bytes
-// inside the 128-byte row, the second 64-column atom after the fourth step).  The issuing
-// thread shares its scheduler with four epilogue warps, so every instruction it saves counts.
-__device__ __forceinline__ void fu_issue_tile(uint32_t tmem, int acc, uint32_t a_base, uint32_t b_base)
+// One 128 x 128 x 128 product into the accumulator at tensor-memory address `d`: eight
+// tcgen05.mma.  `a_lo` / `b_lo` are the start-address fields (shared-memory address / 16) of the
+// operands' descriptors; the rest of a descriptor is constant (128-byte swizzle, eight-row groups
+// 1024 bytes apart, version 1).  A k-step moves the start address by 32 bytes inside the 128-byte
+// row, the second 64-column atom follows after the fourth step.
+__device__ __forceinline__ void fu_issue_tile(uint32_t d, uint32_t a_lo, uint32_t b_lo)
 {
     constexpr uint32_t idesc = umma_idesc_bf16(128, 128);
-    const uint64_t da = umma_desc_sw128(a_base), db = umma_desc_sw128(b_base);
-    const uint32_t d = tmem + (uint32_t)acc * 128u;
-#pragma unroll
-    for (int kk = 0; kk < 8; ++kk) {
-        constexpr uint32_t kAtom16 = kAtomBytes >> 4;
-        const uint32_t off16 = (uint32_t)(kk >> 2) * kAtom16 + (uint32_t)(kk & 3) * 2u;      // byte offset / 16
-        if (kk == 0)
-            asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, 0, 0;\n\t"
-                         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-                         ::"r"(d), "l"(da + off16), "l"(db + off16), "r"(idesc) : "memory");
-        else
-            asm volatile("{\n\t.reg .pred p;\n\tsetp.eq.b32 p, 0, 0;\n\t"
-                         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-                         ::"r"(d), "l"(da + off16), "l"(db + off16), "r"(idesc) : "memory");
-    }
+    constexpr uint32_t desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);     // bits 32-63 of umma_desc_sw128()
+    static_assert((kAtomBytes >> 4) == 1024, "start-address step of the second atom");
+#define FU_MMA_STEP(OFF, PRED)                                                        \
+        "add.u32 ta, %1, " #OFF ";\n\tadd.u32 tb, %2, " #OFF ";\n\t"                  \
+        "mov.b64 da, {ta, %3};\n\tmov.b64 db, {tb, %3};\n\t"                          \
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, " #PRED ";\n\t"
+    asm volatile(
+        "{\n\t.reg .pred yes, no;\n\t.reg .b32 ta, tb;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 no, 0, 0;\n\tsetp.eq.b32 yes, 0, 0;\n\t"
+        FU_MMA_STEP(0, no) FU_MMA_STEP(2, yes) FU_MMA_STEP(4, yes) FU_MMA_STEP(6, yes)
+        FU_MMA_STEP(1024, yes) FU_MMA_STEP(1026, yes) FU_MMA_STEP(1028, yes) FU_MMA_STEP(1030, yes)
+        "}"
+        ::"r"(d), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc)
+        : "memory");
+#undef FU_MMA_STEP
 }
 
 // ---- arithmetic of the epilogue ---------------------------------------------------------------
@@ -839,52 +840,62 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         // blocks for about as long as the tensor core needs for the tile, so everything else this
         // thread does per step is kept short: no state in local memory, barrier probes whose
         // latencies overlap, the next step's record fetched while the products are issued.
+        // It runs at a fraction of an instruction per clock (four epilogue warps share its
+        // scheduler), so the loop keeps its own arithmetic to a minimum: ring positions, parities and
+        // the start-address fields of the descriptors are carried along instead of recomputed.
         if (lane == 0) {
-            int n = 0;
-            int4 e, e_next = make_int4(0, 0, 0, 0);
+            const uint32_t q_lo0 = (q_smem & 0x3FFFFu) >> 4, k_lo0 = (k_smem & 0x3FFFFu) >> 4;    // descriptor start-address fields
+            constexpr uint32_t kTileLo = kFuTileBytes >> 4;
+            const uint32_t bar_full0 = smem_u32(&sh.full[0]), bar_empty0 = smem_u32(&sh.empty[0]);
+            const uint32_t bar_tfull0 = smem_u32(&sh.tfull[0]), bar_tempty0 = smem_u32(&sh.tempty[0]);
+            int n = 0, flags = 0, flags_next = 0;
+            uint32_t st = 0, kpar = 0;                         // K stage of the step and the parity of its fill
             bool have_next = false;
             while (true) {
-                if (have_next) e = e_next;
-                else if (!sched_get(sched, n, e, abort_flag)) break;
-                have_next = false;
-                const int flags = e.x;
-#pragma unroll
-                for (int i = 0; i < kFuQBufs; ++i)
-                    if (flags & (1 << (kStepRelShift + i))) tc_commit(smem_u32(&sh.qempty[i]));
-                const int b = (flags >> kStepQBufShift) & 3;
-                const int acc = n & 1, n_mine = n >> 1;            // accumulator of the step, its uses so far
-                const int st = n % kFuStages, par = (n / kFuStages) & 1;
-                {
-                    FU_TRACE(1, n, 0);
-                    // both barriers are probed before either result is looked at, so that their
-                    // latencies overlap; only a barrier that is not complete yet is waited for
-                    bool te_ok, k_ok;
-                    mbar_test_wait2(smem_u32(&sh.tempty[acc]), (uint32_t)((n_mine & 1) ^ 1), smem_u32(&sh.full[st]), (uint32_t)par,
-                                    te_ok, k_ok);
-                    // the first product that uses a load of the query block waits for it
-                    if ((flags & kStepNewQ) && !FU_WAIT(3, mbar_wait(smem_u32(&sh.qfull[b]), (flags & kStepQPar) ? 1u : 0u, abort_flag))) break;
-                    if (!te_ok && !FU_WAIT(4, mbar_wait(smem_u32(&sh.tempty[acc]), (uint32_t)((n_mine & 1) ^ 1), abort_flag))) break;
-                    FU_TRACE(1, n, 4);
-                    FU_TRACE_VAL(1, n, 5, flags);
-                    if (!k_ok && !FU_WAIT(5, mbar_wait(smem_u32(&sh.full[st]), (uint32_t)par, abort_flag))) break;
-                    FU_TRACE(1, n, 1);
-                    tc_fence_after();
-                    // the next step's record, if it is posted, comes in while the products are issued
-                    if (sched_count(sched) > n + 1) {
-                        const uint32_t src = smem_u32(&sched.ring[(n + 1) % kFuRing]);
-                        asm volatile("ld.volatile.shared.v4.s32 {%0, %1, %2, %3}, [%4];"
-                                     : "=r"(e_next.x), "=r"(e_next.y), "=r"(e_next.z), "=r"(e_next.w) : "r"(src) : "memory");
-                        have_next = true;
-                    }
-                    const uint32_t kt = k_smem + st * kFuTileBytes, qt = q_smem + b * kFuTileBytes;
-                    const bool is_b = (flags & kStepB) != 0;
-                    fu_issue_tile(tmem, acc, is_b ? kt : qt, is_b ? qt : kt);      // rows = tokens (B) or window rows (A)
-                    FU_TRACE(1, n, 2);
-                    tc_commit(smem_u32(&sh.empty[st]));
-                    tc_commit(smem_u32(&sh.tfull[acc]));
-                    FU_TRACE(1, n, 3);
+                if (have_next) {
+                    flags = flags_next;
+                } else {
+                    int4 e;
+                    if (!sched_get(sched, n, e, abort_flag)) break;
+                    flags = e.x;
                 }
+                have_next = false;
+                if (flags & (7 << kStepRelShift)) {
+#pragma unroll
+                    for (int i = 0; i < kFuQBufs; ++i)
+                        if (flags & (1 << (kStepRelShift + i))) tc_commit(smem_u32(&sh.qempty[i]));
+                }
+                const uint32_t b = (uint32_t)(flags >> kStepQBufShift) & 3u;
+                const uint32_t acc = (uint32_t)n & 1u;             // accumulator of the step
+                const uint32_t te_par = (((uint32_t)n >> 1) & 1u) ^ 1u;
+                const uint32_t bar_te = bar_tempty0 + acc * 8u, bar_k = bar_full0 + st * 8u;
+                FU_TRACE(1, n, 0);
+                // both barriers are probed before either result is looked at, so that their
+                // latencies overlap; only a barrier that is not complete yet is waited for
+                bool te_ok, k_ok;
+                mbar_test_wait2(bar_te, te_par, bar_k, kpar, te_ok, k_ok);
+                // the first product that uses a load of the query block waits for it
+                if ((flags & kStepNewQ) && !FU_WAIT(3, mbar_wait(smem_u32(&sh.qfull[b]), (flags & kStepQPar) ? 1u : 0u, abort_flag))) break;
+                if (!te_ok && !FU_WAIT(4, mbar_wait(bar_te, te_par, abort_flag))) break;
+                FU_TRACE(1, n, 4);
+                FU_TRACE_VAL(1, n, 5, flags);
+                if (!k_ok && !FU_WAIT(5, mbar_wait(bar_k, kpar, abort_flag))) break;
+                FU_TRACE(1, n, 1);
+                tc_fence_after();
+                // the next step's flags, if it is posted, come in while the products are issued
+                if (sched_count(sched) > n + 1) {
+                    asm volatile("ld.volatile.shared.s32 %0, [%1];" : "=r"(flags_next) : "r"(smem_u32(&sched.ring[(n + 1) % kFuRing])) : "memory");
+                    have_next = true;
+                }
+                const uint32_t k_lo = k_lo0 + st * kTileLo, q_lo = q_lo0 + b * kTileLo;
+                const bool is_b = (flags & kStepB) != 0;
+                fu_issue_tile(tmem + acc * 128u, is_b ? k_lo : q_lo, is_b ? q_lo : k_lo);   // rows = tokens (B) or window rows (A)
+                FU_TRACE(1, n, 2);
+                tc_commit(bar_empty0 + st * 8u);
+                tc_commit(bar_tfull0 + acc * 8u);
+                FU_TRACE(1, n, 3);
                 ++n;
+                if (++st == kFuStages) { st = 0; kpar ^= 1u; }
             }
         }
     } else if (warp == kFuHelpWarp) {
