@@ -77,6 +77,12 @@ constexpr int kReleaseAt = SABLOCK_RELEASE_AT;
 #define SABLOCK_AHEAD 1
 #endif
 constexpr bool kAhead = SABLOCK_AHEAD != 0;
+#ifndef SABLOCK_XU_PASS_A
+#define SABLOCK_XU_PASS_A 1      // sweep A passes the turn after this many of its two chunks (1 measured best)
+#endif
+#ifndef SABLOCK_XU_PASS_B
+#define SABLOCK_XU_PASS_B 3      // sweep B passes the turn after this many of its four heads (3 measured best)
+#endif
 #ifndef SABLOCK_XU_TURNS
 #define SABLOCK_XU_TURNS 1
 #endif
@@ -84,8 +90,9 @@ constexpr bool kAhead = SABLOCK_AHEAD != 0;
 // unit of the kernel; two sets that share it freely end up in lockstep, both computing and then
 // both going through the latencies between two steps (step record, accumulator barrier,
 // tensor-memory loads) with the unit idle.  With turns, set s starts the exponentials of its k-th
-// step only when the other set is halfway through those of its own preceding step, which keeps
-// the sets half a step apart: while one goes through the latencies the other has the unit.
+// step only when the other set is well into those of its own preceding step (halfway in sweep A,
+// three heads of four in sweep B), which keeps the sets apart: while one goes through the
+// latencies the other has the unit.
 constexpr bool kXuTurns = SABLOCK_XU_TURNS != 0;
 
 struct FusedArgs {
@@ -1098,10 +1105,11 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     if (kXuTurns && !FU_WAIT(9, mbar_wait(smem_u32(&sh.xu[set]), (uint32_t)((n_mine & 1) ^ (set ^ 1)), abort_flag))) break;
                     if (first_thread) FU_TRACE(2 + set, n_mine, 6);
                     rs.add(r0, c2);
-                    if (kXuTurns) mbar_arrive(smem_u32(&sh.xu[set ^ 1]));
+                    if (kXuTurns && SABLOCK_XU_PASS_A == 1) mbar_arrive(smem_u32(&sh.xu[set ^ 1]));
                     if (kReleaseAt == 1) mbar_arrive(smem_u32(&sh.tempty[set]));
                     if (kAhead) ahead_flags = sched_peek_flags(sched, set, n_mine + 1);
                     rs.add(r1, c2);
+                    if (kXuTurns && SABLOCK_XU_PASS_A == 2) mbar_arrive(smem_u32(&sh.xu[set ^ 1]));
                     if (kAhead) ahead_tfull = mbar_test_wait(smem_u32(&sh.tfull[set]), (uint32_t)((n_mine + 1) & 1));
                     if (kReleaseAt == 2) mbar_arrive(smem_u32(&sh.tempty[set]));
                     if (first_thread) FU_TRACE(2 + set, n_mine, 7);
@@ -1136,12 +1144,15 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     if (kXuTurns && !FU_WAIT(9, mbar_wait(smem_u32(&sh.xu[set]), (uint32_t)((n_mine & 1) ^ (set ^ 1)), abort_flag))) break;
                     if (first_thread) FU_TRACE(2 + set, n_mine, 6);
                     accumulate_head16(accw, v0, lj, c2);
+                    if (kXuTurns && SABLOCK_XU_PASS_B == 1) mbar_arrive(smem_u32(&sh.xu[set ^ 1]));
                     accumulate_head16(accw, v1, lj + 32, c2);
-                    if (kXuTurns) mbar_arrive(smem_u32(&sh.xu[set ^ 1]));
+                    if (kXuTurns && SABLOCK_XU_PASS_B == 2) mbar_arrive(smem_u32(&sh.xu[set ^ 1]));
                     if (kReleaseAt == 1) mbar_arrive(smem_u32(&sh.tempty[set]));
                     if (kAhead) ahead_flags = sched_peek_flags(sched, set, n_mine + 1);
                     accumulate_head16(accw, v2, lj + 64, c2);
+                    if (kXuTurns && SABLOCK_XU_PASS_B == 3) mbar_arrive(smem_u32(&sh.xu[set ^ 1]));
                     accumulate_head16(accw, v3, lj + 96, c2);
+                    if (kXuTurns && SABLOCK_XU_PASS_B == 4) mbar_arrive(smem_u32(&sh.xu[set ^ 1]));
                     if (kAhead) ahead_tfull = mbar_test_wait(smem_u32(&sh.tfull[set]), (uint32_t)((n_mine + 1) & 1));
                     if (kReleaseAt == 2) mbar_arrive(smem_u32(&sh.tempty[set]));
                     if (first_thread) FU_TRACE(2 + set, n_mine, 7);
