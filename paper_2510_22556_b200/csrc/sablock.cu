@@ -438,6 +438,12 @@ sablock_status_t run_score(const Plan& pl, const sablock_params_t* p, const void
 }
 
 // Stage 3 (with optional pooling first): s_raw -> s (pooled) -> s_refined.
+#ifndef SABLOCK_SEG_GRID_PER_2K
+#define SABLOCK_SEG_GRID_PER_2K 8
+#endif
+constexpr int kSegGridPer2K = SABLOCK_SEG_GRID_PER_2K;   // CTAs of the per-segment kernels per 2048 tokens of a sequence
+constexpr int kSegGridMax = 32 * kSegGridPer2K;
+
 sablock_status_t run_refine(const Plan& pl, const sablock_params_t* p, const float* s_raw, float* s, const float* e,
                             const int* seg_start, const int* n_seg, float* s_ref, float* stats, int stats_stride,
                             cudaStream_t stream)
@@ -447,7 +453,10 @@ sablock_status_t run_refine(const Plan& pl, const sablock_params_t* p, const flo
         pool_kernel<<<dim3(gx * 4, pl.n_prob), 256, 0, stream>>>(pl.geo, s_raw, s, p->pool_kernel, p->pool_mode);
         SAB_TRY(check_launch());
     }
-    refine_kernel<<<dim3(gx, pl.n_prob), 256, 0, stream>>>(pl.geo, s, e, seg_start, n_seg, p->alpha, p->eta, s_ref,
+    // one warp per segment, a few dependent loads each: the kernel is latency-bound, so it gets
+    // enough warps to keep every SM's warp slots full (about ten segments per warp)
+    const int gr = (int)fmin((double)kSegGridMax, fmax(1.0, (double)((pl.max_L + 2047) / 2048) * kSegGridPer2K));
+    refine_kernel<<<dim3(gr, pl.n_prob), 256, 0, stream>>>(pl.geo, s, e, seg_start, n_seg, p->alpha, p->eta, s_ref,
                                                            stats, stats_stride);
     return check_launch();
 }
@@ -508,7 +517,7 @@ sablock_status_t run_select(const Plan& pl, const sablock_params_t* p, const flo
     so.long_list = at<int>(ws, pl.o_long_list);
     so.long_count = at<int>(ws, pl.o_long_count);
     so.long_cap = pl.long_cap;
-    const int gx = (int)fmin(32.0, fmax(1.0, (double)((pl.max_L + 2047) / 2048)));
+    const int gx = (int)fmin((double)kSegGridMax, fmax(1.0, (double)((pl.max_L + 2047) / 2048) * kSegGridPer2K));
     search_kernel<<<dim3(gx, pl.n_prob), kSearchWarps * 32, 0, stream>>>(g, cands, s_ref, seg_start, n_seg, thr, cut,
                                                                         p->tau, so);
     SAB_TRY(check_launch());

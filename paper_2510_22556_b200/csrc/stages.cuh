@@ -440,12 +440,12 @@ search_kernel(Geo g, Cands cands, const float* __restrict__ s_ref, const int* __
             if (in_topb(v, a + i, thr, cut)) { ++b; base += (double)v; }
         }
         b = warp_sum(b);
-        base = warp_sum(base);
         if (out.seg_b && lane == 0) out.seg_b[(size_t)p * out.seg_stride + k] = b;
-        if (b == 0) {
+        if (b == 0) {                               // most segments at small budgets: nothing to search
             if (out.seg_g && lane == 0) out.seg_g[(size_t)p * out.seg_stride + k] = 0;
             continue;
         }
+        base = warp_sum(base);
         if (n > kSegShort) {
             if (lane == 0) {
                 int slot = atomicAdd(&out.long_count[p], 1);
