@@ -383,8 +383,10 @@ def run_ours_isolated():
         tail = [l for l in proc.stderr.splitlines() if l.strip()][-1:] or ["no message"]
         faults.append(tail[0][:300])
         sys.stderr.write(proc.stderr)
-        is_cuda_fault = "CUDA" in proc.stderr
-        if not is_cuda_fault:
+        # only a device fault of a run that had a GPU is worth another attempt
+        is_device_fault = any(t in proc.stderr for t in ("launch failure", "illegal memory access", "illegal instruction",
+                                                         "CUDA runtime or driver error", "AcceleratorError"))
+        if not is_device_fault:
             break
     sys.stderr.write("bench.py: no successful measurement in %d attempt(s)\n" % len(faults))
     sys.exit(1)
