@@ -737,7 +737,9 @@ sablock_status_t sablock_score(const sablock_params_t* p, const void* q_win, con
     t_launches = 0;
     if (!p || L <= p->window || !seg_start || !n_seg || !s || !s_refined) return SABLOCK_ERR_INVALID_ARG;
     Plan pl;
-    SAB_TRY(make_plan(p, 1, 1, nullptr, L, L, p->window + 1, &pl));
+    // no budget here: "output rows" = the window alone, so that no sequence with a compressible
+    // token (L > W) counts as one that is returned unchanged
+    SAB_TRY(make_plan(p, 1, 1, nullptr, L, L, p->window, &pl));
     if (!ws || ws_bytes < pl.total) return SABLOCK_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     SAB_TRY(zero_control(pl, ws, st));

@@ -114,6 +114,54 @@ def test_score_tensor_core_heavy_tails():
     _score_case(32, 8, 128, 32, 3000, torch.bfloat16, B.SCORE_TENSOR, 9, kappa=6.0)
 
 
+@pytest.mark.parametrize("H,Hkv,L", [
+    (32, 8, 8192),         # Llama-3-8B shape, 64 tiles: fewer tiles than CTAs
+    (32, 8, 4096 + 55),    # ragged tail, window straddles a tile boundary
+    (32, 8, 20000),        # more tiles than CTAs: some CTAs hold two
+    (8, 2, 160),           # two tiles only
+    (8, 2, 129),           # T < one tile; the second tile holds window keys only
+    (8, 2, 128),           # one tile in all: 96 compressible tokens and the window
+    (4, 1, 128 * 3 + 32),  # T a whole number of tiles: the window has a tile of its own
+])
+def test_score_fused_bf16(H, Hkv, L):
+    _score_case(H, Hkv, 128, 32, L, torch.bfloat16, B.SCORE_FUSED, L + 3)
+
+
+def test_score_fused_heavy_tails():
+    # large logits: the row sums' reference exponents must move without losing the sum
+    _score_case(32, 8, 128, 32, 3000, torch.bfloat16, B.SCORE_FUSED, 9, kappa=6.0)
+
+
+def test_score_fused_agrees_with_two_launch_path():
+    # two implementations of the same arithmetic up to the order of the fp32 sums
+    cfg = synth.Config("t", 1, 32, 8, 128, 32, (6000,), (64,), (1, 2), "bf16", 128256, 8, 2.0, 25, (0.4,), 21)
+    q, k, v, _ = synth.make_layer(cfg, 6000, 21)
+    ids = synth.make_token_ids(6000, cfg.vocab, 25, 22)
+    bm = synth.delimiter_bitmap(cfg.vocab).cuda()
+    outs = []
+    for impl in (B.SCORE_FUSED, B.SCORE_TENSOR):
+        p = B.make_params(32, 8, 128, 32, torch.bfloat16, bm, cfg.vocab, score_impl=impl)
+        ws = B.alloc_workspace(p, 6000, 6000)
+        _, seg_start, n_seg = B.segment(p, ids.cuda(), ws)
+        s, e, sr, _ = B.score(p, q.cuda(), k.cuda(), seg_start, n_seg, ws)
+        _sync_ok(ws)
+        outs.append((s.double().cpu().numpy(), e.double().cpu().numpy()))
+    (s0, e0), (s1, e1) = outs
+    assert np.abs(s0 - s1).max() <= 1e-7 + 2e-5 * np.abs(s1).max()
+    assert np.abs(e0 - e1).max() <= 1e-4
+
+
+def test_score_fused_refuses_what_it_cannot_run():
+    bm = synth.delimiter_bitmap(128256).cuda()
+    p = B.make_params(16, 4, 64, 32, torch.bfloat16, bm, 128256, score_impl=B.SCORE_FUSED)     # head_dim 64
+    with pytest.raises(B.SablockError):
+        B.alloc_workspace(p, 4096, 4096)
+    # fewer key rows than one 128-row TMA box: forced FUSED says so, AUTO takes the SIMT kernels
+    with pytest.raises(B.SablockError):
+        _score_case(8, 2, 128, 32, 33, torch.bfloat16, B.SCORE_FUSED, 5)
+    _score_case(8, 2, 128, 32, 33, torch.bfloat16, B.SCORE_AUTO, 5)
+
+
 @pytest.mark.parametrize("pool", [(7, 0), (7, 1), (3, 1)])
 def test_score_with_pooling(pool):
     _score_case(32, 8, 128, 32, 2000, torch.bfloat16, B.SCORE_AUTO, 4, pool=pool)
