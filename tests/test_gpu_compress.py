@@ -182,6 +182,44 @@ def test_host_buffer_entry_point():
     assert torch.equal(h_out.out_v, ref.out_v.cpu()) and h_out.n_keep.tolist() == [[128, 128]] * 2
 
 
+@pytest.mark.parametrize("L,budget", [
+    (2000, 33),        # B = 1: one token besides the window
+    (2000, 34),
+    (2000, 1999),      # B = T - 1: all but one
+    (2000, 2000),      # budget = L: returned unchanged
+    (2000, 2100),      # budget > L
+    (33, 33),          # a single compressible token, and it fits
+    (160, 100),        # two score tiles
+    (4096, 4000),      # nearly everything kept, Llama shape through the persistent kernel
+])
+def test_budget_extremes(L, budget):
+    cfg = synth.CONFIGS["layer8k"]
+    b = synth.make_batch(cfg, device="cuda", seq_lens=[L])
+    out, infos = run_batch(cfg, b, budget)
+    assert out.n_keep.item() == min(budget, L)
+
+
+def test_sequence_lengths_around_tile_boundaries():
+    # one batch whose sequences end just before, at and just after multiples of the 128-token tile
+    cfg = synth.CONFIGS["ragged16"]
+    lens = [128 * 3 - 1, 128 * 3, 128 * 3 + 1, 128 * 3 + 31, 128 * 3 + 32, 128 * 3 + 33, 1024 + 32]
+    b = synth.make_batch(cfg, device="cuda", n_layers=2, seq_lens=lens)
+    out, infos = run_batch(cfg, b, 96)
+    assert out.n_keep.cpu().tolist() == [[96] * len(lens)] * 2
+
+
+def test_longest_sequence_of_the_persistent_kernel_and_beyond():
+    """7 tiles per CTA x 148 CTAs x 128 tokens is the most the persistent score kernel takes on
+    B200; one tile more goes to the two-launch kernels.  Same protocol, one layer each."""
+    cfg = synth.CONFIGS["headline128k"]
+    for L in (7 * 148 * 128, 7 * 148 * 128 + 128):
+        b = synth.make_batch(cfg, device="cuda", n_layers=1, seq_lens=[L])
+        out, infos = run_batch(cfg, b, 1024)
+        assert out.n_keep.item() == 1024
+        del b, out
+        torch.cuda.empty_cache()
+
+
 def test_headline_config_full_size():
     """The benchmark's launch configuration: 32 layers x 131072 tokens, budget 1024.  Layers 0 and
     31 are checked against the oracle in full; every layer is checked for the invariants."""
