@@ -237,7 +237,7 @@ def run_ours(args):
 
 # DRAM bytes (read + write) per launch from the ncu capture summarised under profiles/,
 # taken on a smaller case and scaled by (layers x tokens); None until captured.
-TRAFFIC_BYTES_PER_LAUNCH = {"score_fused_tc": 554024704}     # profiles/score_fused_tc_headline128k_2layers.txt
+TRAFFIC_BYTES_PER_LAUNCH = {"score_fused_tc": 554110720}     # profiles/score_fused_tc_headline128k_2layers.txt
 TRAFFIC_CAPTURE_TOKEN_LAYERS = 2 * 131072
 
 
