@@ -366,6 +366,8 @@ MAX_ATTEMPTS = 3
 
 def run_ours_isolated():
     import subprocess
+    from paper_2510_22556_b200 import binding as B
+    B.lib()          # fails loudly, here already, if the CUDA library is missing: there is no fallback
     faults = []
     for attempt in range(1, MAX_ATTEMPTS + 1):
         env = dict(os.environ)
