@@ -485,7 +485,11 @@ sablock_status_t run_select(const Plan& pl, const sablock_params_t* p, const flo
         int ctas = 1;
         int dev = 0, sms = 0;
         if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0) {
-            ctas = sms / pl.n_prob;
+            // all CTAs of the launch must be co-resident: as many per SM as the kernel's occupancy allows
+            int per_sm = 1;
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, topb_kernel, kTopThreads, 0) != cudaSuccess || per_sm < 1)
+                per_sm = 1;
+            ctas = sms * per_sm / pl.n_prob;
             const int by_len = (pl.max_L + 4 * kTopThreads - 1) / (4 * kTopThreads);      // at least four rounds each
             if (ctas > by_len) ctas = by_len;
             if (ctas > kTopMaxCtas) ctas = kTopMaxCtas;
