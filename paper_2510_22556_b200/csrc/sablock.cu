@@ -546,7 +546,7 @@ sablock_status_t run_compact(const Geo& g, int n_prob, const sablock_params_t* p
     c.k_tok = ks.tok * es; c.k_head = ks.head * es; c.k_layer = ks.layer * es;
     c.v_tok = vs.tok * es; c.v_head = vs.head * es; c.v_layer = vs.layer * es;
     c.head_bytes = g.D * es;
-    c.rows_per_cta = 4;
+    c.rows_per_cta = (long long)g.n_out * n_prob >= 16384 ? 8 : 4;     // larger CTAs once there are thousands of them
     const long long all[] = {c.k_tok, c.k_head, c.k_layer, c.v_tok, c.v_head, c.v_layer};
     for (long long x : all)
         if (x % 16) return SABLOCK_ERR_UNSUPPORTED;
