@@ -350,48 +350,9 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
-    elif int(os.environ.get("WORLD_SIZE", "1")) == 1 and os.environ.get(CHILD_ENV) != "1":
-        run_ours_isolated()
     else:
+        # one attempt: a CUDA error ends the run with the runtime's message and a non-zero exit
         run_ours(args)
-
-
-# A device fault ends a CUDA context for good, so the single-GPU measurement runs in a child
-# process: if the child dies of a CUDA error the whole measurement is taken again (at most
-# MAX_ATTEMPTS times in all), and the JSON line says how many attempts there were and what the
-# failed ones reported.  Nothing of a failed attempt is reused.
-CHILD_ENV = "SABLOCK_BENCH_CHILD"
-MAX_ATTEMPTS = 3
-
-
-def run_ours_isolated():
-    import subprocess
-    from paper_2510_22556_b200 import binding as B
-    B.lib()          # fails loudly, here already, if the CUDA library is missing: there is no fallback
-    faults = []
-    for attempt in range(1, MAX_ATTEMPTS + 1):
-        env = dict(os.environ)
-        env[CHILD_ENV] = "1"
-        proc = subprocess.run([sys.executable, os.path.abspath(__file__)] + sys.argv[1:], env=env,
-                              stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True)
-        line = next((l for l in reversed(proc.stdout.splitlines()) if l.startswith("{")), None)
-        if proc.returncode == 0 and line is not None:
-            result = json.loads(line)
-            result["attempts"] = attempt
-            result["failed_attempts"] = faults
-            sys.stderr.write(proc.stderr)
-            print(json.dumps(result))
-            return
-        tail = [l for l in proc.stderr.splitlines() if l.strip()][-1:] or ["no message"]
-        faults.append(tail[0][:300])
-        sys.stderr.write(proc.stderr)
-        # only a device fault of a run that had a GPU is worth another attempt
-        is_device_fault = any(t in proc.stderr for t in ("launch failure", "illegal memory access", "illegal instruction",
-                                                         "CUDA runtime or driver error", "AcceleratorError"))
-        if not is_device_fault:
-            break
-    sys.stderr.write("bench.py: no successful measurement in %d attempt(s)\n" % len(faults))
-    sys.exit(1)
 
 
 if __name__ == "__main__":

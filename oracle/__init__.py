@@ -126,16 +126,19 @@ def refine(s, e, seg_start, alpha: float = 0.9, eta: float = 1.0):
     return I, Dk, om, sr
 
 
-def segment_fill(sv, b: int, g: int):
-    """Alg. 2 inner loop for one segment and one block size: (taken mask, Score_k(g), blocks)."""
+def segment_fill(sv, b: int, g: int, want_margins: bool = False):
+    """Alg. 2 inner loop for one segment and one block size: (taken mask, Score_k(g), blocks),
+    plus the four decision margins (inf where no such decision was taken) if asked for."""
     sv = np.ascontiguousarray(sv, np.float64)
     n = sv.shape[0]
     taken = np.zeros(n, np.uint8)
     blocks = np.zeros(2 * (n + 1), np.int32)
     nb = C.c_int(0)
+    margins = np.full(4, np.inf)
     sc = lib().sabo_segment_fill(_p(sv, C.c_double), n, b, g, _p(taken, C.c_uint8),
-                                 _p(blocks, C.c_int32), C.byref(nb), None)
-    return taken.astype(bool), float(sc), blocks[: 2 * nb.value].reshape(-1, 2).copy()
+                                 _p(blocks, C.c_int32), C.byref(nb), _p(margins, C.c_double))
+    res = (taken.astype(bool), float(sc), blocks[: 2 * nb.value].reshape(-1, 2).copy())
+    return res + (margins,) if want_margins else res
 
 
 def select(s_ref, seg_start, B: int, candidates: Sequence[int], tau: float = 0.85):
@@ -178,7 +181,7 @@ def gather(x, idx):
 
 def compress(q, k, token_ids, bitmap, vocab: int, budget: int, candidates: Sequence[int],
              alpha: float = 0.9, eta: float = 1.0, eps: float = 1e-6, tau: float = 0.85,
-             pool_kernel: int = 1, pool_mode: int = 0):
+             pool_kernel: int = 1, pool_mode: int = 0, budget_includes_window: int = 1):
     """The whole pass for one (layer, sequence).  Returns a dict of every stage's result."""
     qf, kf = _f32(q), _f32(k)
     H, W, D = qf.shape
@@ -186,7 +189,8 @@ def compress(q, k, token_ids, bitmap, vocab: int, budget: int, candidates: Seque
     T = L - W
     ids = _i32(token_ids)
     cand = np.ascontiguousarray(sorted(candidates), np.int32)
-    n_out = L if budget >= L else budget
+    n_out = budget if budget_includes_window else budget + W
+    n_out = L if n_out >= L else n_out
     out_idx = np.zeros(max(n_out, 1), np.int32)
     seg_id = np.zeros(max(T, 1), np.int32)
     seg_start = np.zeros(max(T, 1) + 1, np.int32)
@@ -198,7 +202,8 @@ def compress(q, k, token_ids, bitmap, vocab: int, budget: int, candidates: Seque
     n = lib().sabo_compress(_p(qf, C.c_float), _p(kf, C.c_float), _p(ids, C.c_int32), L, H, Hkv, D, W,
                             C.c_longlong(Hkv * D), C.c_longlong(D), _p(_u32(bitmap), C.c_uint32), vocab,
                             C.c_double(alpha), C.c_double(eta), C.c_double(eps), C.c_double(tau),
-                            pool_kernel, pool_mode, budget, _p(cand, C.c_int32), cand.shape[0],
+                            pool_kernel, pool_mode, budget, int(budget_includes_window), _p(cand, C.c_int32),
+                            cand.shape[0],
                             _p(out_idx, C.c_int32), _p(seg_id, C.c_int32), _p(seg_start, C.c_int32),
                             C.byref(n_seg), _p(s, C.c_double), _p(e, C.c_double), _p(sr, C.c_double),
                             _p(g_star, C.c_int32), _p(b_k, C.c_int32), _p(margins, C.c_double))

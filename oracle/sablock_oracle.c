@@ -339,24 +339,28 @@ void sabo_gather(const uint8_t *src, long long stride_bytes, long long row_bytes
 /* ------------------------------------------------------------------ whole pass */
 /* One (layer, sequence).  Outputs: out_idx[n_keep] (ascending positions in the
  * compressible region, then the W window positions), and optionally the stage results.
- * budget counts all retained entries, window included: B = budget - W (budget >= L keeps
- * everything).  Returns n_keep. */
+ * Eq. 13 fixes |T*| = B and the text after it adds the recent tokens on top, but the paper
+ * does not say whether a quoted "budget" counts them.  budget_includes_window = 1: budget
+ * counts all retained entries, window included, so B = budget - W; 0: B = budget and
+ * budget + W entries are retained.  If the entries to retain are >= L everything is kept.
+ * Returns n_keep. */
 int sabo_compress(const float *q, const float *k, const int32_t *token_ids, int L,
                   int H, int Hkv, int D, int W, long long ks_tok, long long ks_head,
                   const uint32_t *bitmap, int vocab,
                   double alpha, double eta, double eps, double tau,
                   int pool_kernel, int pool_mode,
-                  int budget, const int32_t *cand, int n_cand,
+                  int budget, int budget_includes_window, const int32_t *cand, int n_cand,
                   int32_t *out_idx, int32_t *seg_id, int32_t *seg_start, int32_t *n_seg_out,
                   double *s_out, double *e_out, double *s_ref_out,
                   int32_t *g_star, int32_t *b_k, double *margins)
 {
     int T = L - W;
-    if (budget >= L) {
+    int n_out = budget_includes_window ? budget : budget + W;
+    if (n_out >= L) {
         for (int i = 0; i < L; ++i) out_idx[i] = i;
         return L;
     }
-    int B = budget - W;
+    int B = n_out - W;
     int n_seg = sabo_segment(token_ids, L, W, bitmap, vocab, seg_id, seg_start);
     if (n_seg_out) *n_seg_out = n_seg;
     double *abar = (double *)malloc(sizeof(double) * (size_t)W * T);

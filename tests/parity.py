@@ -2,10 +2,11 @@
 
 Scores: |gpu - ref| <= ABS + REL * |ref| with the tolerance the benchmark spec states for bf16 inputs
 with fp32 accumulation (rel 2e-3, abs 1e-5).  Integer results (segment ids, indices, block
-sizes) and K/V bytes: bit-exact.  Where the oracle's float64 scores make a decision on a gap
-smaller than the score tolerance, the index comparison is tie-aware: Algorithm 2 is re-run
-by the oracle on the GPU's own fp32 refined scores and must reproduce the GPU's indices
-exactly.
+sizes) and K/V bytes: bit-exact.  Only where the oracle's float64 scores make a decision on a
+relative gap smaller than the score tolerance REL may the indices differ from the pure oracle's;
+then the comparison is tie-aware: Algorithm 2 is re-run by the oracle on the GPU's own fp32
+refined scores and must reproduce the GPU's indices exactly, and the retained score mass must
+agree with the pure oracle's within the same tolerance.
 """
 from __future__ import annotations
 
@@ -45,6 +46,8 @@ def check_problem(cfg_like, q, k, v, ids, bitmap, vocab, budget, candidates, out
     assert int(n_keep) == n_ref, ("n_keep", int(n_keep), n_ref)
     idx = out_idx[:n_ref].detach().cpu().numpy()
     info = dict(n_keep=n_ref, margins=r["margins"].copy())
+    if n_ref < L and (r["b_k"] > 0).any():
+        info["mean_g"] = float(r["g_star"][r["b_k"] > 0].mean())
     if n_ref < L:
         if s_gpu is not None:
             info["s_relerr"] = assert_scores_close(s_gpu[:T], r["s"], "s")
@@ -60,7 +63,7 @@ def check_problem(cfg_like, q, k, v, ids, bitmap, vocab, budget, candidates, out
         if not exact:
             # tie-aware: allowed only if some decision margin of the pure oracle is below tolerance,
             # and Algorithm 2 on the GPU's own refined scores reproduces the GPU's indices exactly.
-            assert r["margins"].min() <= 4 * REL, ("indices differ although every margin is wide", r["margins"])
+            assert r["margins"].min() < REL, ("indices differ although every margin is wide", r["margins"])
             assert sr_gpu is not None, "need the GPU's refined scores for the tie-aware check"
         if sr_gpu is not None:
             B = n_ref - W
@@ -70,7 +73,7 @@ def check_problem(cfg_like, q, k, v, ids, bitmap, vocab, budget, candidates, out
             # retained refined-score mass within tolerance of the pure oracle's
             mass_gpu = r["s_ref"][idx[:B]].sum()
             mass_ref = r["s_ref"][r["out_idx"][:B]].sum()
-            assert abs(mass_gpu - mass_ref) <= 4 * REL * mass_ref + ABS
+            assert abs(mass_gpu - mass_ref) <= REL * mass_ref + ABS
     else:
         assert idx.tolist() == list(range(L))
     # compaction: byte-exact gather at the (validated) indices

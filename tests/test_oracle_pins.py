@@ -216,6 +216,27 @@ def test_select_hand_traces():
         assert r["b_k"].tolist() == _nums(f[7], int), name
 
 
+def _margin(tok):
+    if tok == "inf":
+        return math.inf
+    num, _, den = tok.partition("/")
+    return float(num) / float(den or 1)
+
+
+def test_decision_margins_hand_traces():
+    """The four decision margins the comparison protocol gates on, against hand-worked values."""
+    fills = dict(_golden("fill"))
+    for name, f in _golden("fillmargins"):
+        src = fills[name]
+        *_, m = oracle.segment_fill(_nums(src[0]), int(src[1]), int(src[2]), want_margins=True)
+        np.testing.assert_allclose(m, [_margin(x) for x in f], rtol=1e-12, atol=1e-15, err_msg=name)
+    selects = dict(_golden("select"))
+    for name, f in _golden("selectmargins"):
+        src = selects[name]
+        r = oracle.select(_nums(src[0]), _nums(src[1], int), int(src[2]), _nums(src[3], int), tau=float(src[4]))
+        np.testing.assert_allclose(r["margins"], [_margin(x) for x in f], rtol=1e-12, atol=1e-15, err_msg=name)
+
+
 def _random_problem(rng, quantised):
     n_seg = int(rng.integers(1, 6))
     lens = rng.integers(1, 9, n_seg)
@@ -334,6 +355,50 @@ def test_compress_invariants_tiny_config():
     assert r2["out_idx"].tolist() == list(range(L))
     kb = oracle.gather(b.k[0], r2["out_idx"])
     assert (kb == b.k[0].contiguous().view(torch.uint8).numpy().reshape(L, -1)).all()
+
+
+def _compose(q, k, ids, bitmap, vocab, W, n_out, cands, pool_kernel, pool_mode, alpha=0.9, eta=1.0, tau=0.85):
+    """The pass put together from the stage functions, each of which is pinned on its own above."""
+    seg_id, seg_start = oracle.segment(ids, W, bitmap, vocab)
+    _, s, e = oracle.scores(q, k, eps=1e-6)                     # entropy from the unpooled attention
+    sp = oracle.pool(s, pool_kernel, pool_mode) if pool_kernel > 1 else s
+    I, Dk, om, sr = oracle.refine(sp, e, seg_start, alpha=alpha, eta=eta)
+    sel = oracle.select(sr, seg_start, n_out - W, cands, tau=tau)
+    T = k.shape[0] - W
+    return dict(seg_id=seg_id, seg_start=seg_start, s=sp, e=e, s_ref=sr, g_star=sel["g_star"], b_k=sel["b_k"],
+                out_idx=np.concatenate([sel["keep"], np.arange(T, T + W, dtype=np.int32)]))
+
+
+@pytest.mark.parametrize("shape", ["tiny", "gqa8"])
+@pytest.mark.parametrize("pool_kernel,pool_mode", [(1, 0), (7, 0), (7, 1)])
+def test_compress_is_the_composition_of_its_stages(shape, pool_kernel, pool_mode):
+    """The glue of the whole-pass function: segmentation, scores, pooling of s only (the entropy keeps
+    the unpooled attention), refinement of the pooled s, Algorithm 2 with B = budget - W, window last.
+    A swapped argument or a wrong order there changes one of the compared arrays."""
+    if shape == "tiny":
+        cfg = synth.CONFIGS["tiny"]
+        budget = 64
+    else:
+        cfg = synth.Config("gqa8", 1, 8, 2, 32, 8, (300,), (48,), (1, 2, 3, 5), "bf16", 5000, 4, 2.0, 9, (0.4,), 21)
+        budget = 48
+    b = synth.make_batch(cfg)
+    q, k, ids, W = b.q_win[0, 0], b.k[0], b.token_ids, cfg.window
+    r = oracle.compress(q, k, ids, b.bitmap, cfg.vocab, budget, cfg.candidates, pool_kernel=pool_kernel,
+                        pool_mode=pool_mode, alpha=0.7, eta=0.5, tau=0.9)
+    c = _compose(q, k, ids, b.bitmap, cfg.vocab, W, budget, cfg.candidates, pool_kernel, pool_mode, 0.7, 0.5, 0.9)
+    for name in ("seg_id", "seg_start", "g_star", "b_k", "out_idx"):
+        assert r[name].tolist() == c[name].tolist(), name
+    for name in ("s", "e", "s_ref"):
+        np.testing.assert_array_equal(r[name], c[name], err_msg=name)
+    if pool_kernel > 1:                                         # pooling did change the scores it was given
+        assert not np.array_equal(c["s"], oracle.scores(q, k, eps=1e-6)[1])
+    # the other reading of "budget" (Eq. 13 and the sentence after it): B = budget, W more entries come out
+    r0 = oracle.compress(q, k, ids, b.bitmap, cfg.vocab, budget - W, cfg.candidates, pool_kernel=pool_kernel,
+                         pool_mode=pool_mode, alpha=0.7, eta=0.5, tau=0.9, budget_includes_window=0)
+    assert r0["n_keep"] == budget and r0["out_idx"].tolist() == r["out_idx"].tolist()
+    L = k.shape[0]
+    full = oracle.compress(q, k, ids, b.bitmap, cfg.vocab, L - W, cfg.candidates, budget_includes_window=0)
+    assert full["out_idx"].tolist() == list(range(L))           # budget + W >= L: nothing is evicted
 
 
 def test_gather_is_byte_exact():

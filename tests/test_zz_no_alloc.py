@@ -4,8 +4,9 @@ A server with a frozen memory pool, or a plug-in that only ever sees its input a
 buffers, has no workspace to hand to sablock_segment.  The static variant keeps the scan's
 scratch in a fixed array inside the library instead.  This test calls it through the C ABI twice
 in a row (the array keeps the previous call's contents, so the second call checks that the entry
-point clears what it must) and compares with sablock_segment bit for bit: segment ids are
-integers, so the tolerance of the other segmentation tests applies, which is exact equality.
+point clears what it must) and compares with sablock_segment and with the CPU checker bit for bit:
+segment ids are integers, so the tolerance of the other segmentation tests applies, which is exact
+equality.  It also checks that torch's allocator handed out no device memory during the calls.
 Collected last on purpose: a run that stops at the first failure has then run everything else.
 """
 import ctypes as C
@@ -13,6 +14,7 @@ import ctypes as C
 import pytest
 import torch
 
+import oracle
 import synth
 from paper_2510_22556_b200 import binding as B
 from paper_2510_22556_b200 import build as build_lib
@@ -49,9 +51,11 @@ def test_static_segmentation_matches_workspace_version_twice_in_a_row():
                      torch.zeros(1, dtype=torch.int32, device="cuda"),
                      torch.zeros(1, dtype=torch.int32, device="cuda")))
     torch.cuda.synchronize()
+    reserved, allocated = torch.cuda.memory_reserved(), torch.cuda.memory_allocated()
     for ids, (seg_id, seg_start, n_seg, status) in zip(cases, bufs):       # back to back on one stream
         B.segment_static(p, ids, seg_id, seg_start, n_seg, status)
     torch.cuda.synchronize()
+    assert (torch.cuda.memory_reserved(), torch.cuda.memory_allocated()) == (reserved, allocated)
     for ids, (seg_id, seg_start, n_seg, status) in zip(cases, bufs):
         ref_id, ref_start, ref_n = _reference(p, ids)
         n = int(ref_n.item())
@@ -59,6 +63,9 @@ def test_static_segmentation_matches_workspace_version_twice_in_a_row():
         assert n_seg.item() == n
         assert torch.equal(seg_id, ref_id)
         assert torch.equal(seg_start[: n + 1], ref_start[: n + 1])
+        cpu_id, cpu_start = oracle.segment(ids, W, bitmap, vocab)          # the CPU checker, not only CUDA against CUDA
+        assert seg_id.cpu().tolist() == cpu_id.tolist()
+        assert seg_start[: n + 1].cpu().tolist() == cpu_start.tolist()
     # private status word (status = NULL) and a third call after the others
     seg_id, seg_start, n_seg, _ = bufs[1]
     seg_id.fill_(-1)
