@@ -44,10 +44,11 @@ typedef enum {
 typedef enum { SABLOCK_F32 = 0, SABLOCK_BF16 = 1 } sablock_dtype_t;
 
 /* Which kernel family computes the attention scores.  AUTO picks, in this order, the
- * persistent two-sweep tensor-core kernel (bf16, head_dim 128, window 32, four query heads
- * per KV head, at most 7 token tiles of 128 per CTA), the two-launch tensor-core kernels
- * (bf16, head_dim 64/128, window 8/16/32), and the SIMT kernels otherwise.  FUSED and TENSOR
- * force the first and the second and fail with SABLOCK_ERR_UNSUPPORTED where they cannot run. */
+ * persistent tensor-core kernel (bf16, head_dim 128, window 32, four query heads per KV head,
+ * at most 7 token tiles of 128 per CTA; two sweeps over K, or one when row_lse is given), the
+ * two-launch tensor-core kernels (bf16, head_dim 64/128, window 8/16/32), and the SIMT kernels
+ * otherwise (with row_lse these run their second pass only).  FUSED and TENSOR force the first
+ * and the second and fail with SABLOCK_ERR_UNSUPPORTED where they cannot run. */
 typedef enum { SABLOCK_SCORE_AUTO = 0, SABLOCK_SCORE_SIMT = 1, SABLOCK_SCORE_TENSOR = 2, SABLOCK_SCORE_FUSED = 3 }
     sablock_score_impl_t;
 
@@ -80,8 +81,18 @@ typedef struct sablock_params {
     const unsigned *delim_bitmap;  /* dev: bit (id % 32) of word (id / 32) set <=> id delimits  */
     int vocab_size;                /* ids outside [0, vocab_size) never delimit                 */
     int score_impl;                /* sablock_score_impl_t                                      */
-    int l2_lag_tiles;              /* tuning knob of the tensor-core score kernel; 0 = default  */
-    int reserved[7];
+    int reserved0;
+    /* Optional, dev f32 [n_layers, n_seqs, H, W] (single-problem calls: [H, W]), or NULL.
+     * row_lse[h][w] = ln sum_{j <= T+w} exp(q_{h,w} . k_j / sqrt(D)): the log of the softmax
+     * normaliser of Eq. 2 for the query at position T + w, over its causal keys, as the prefill's
+     * attention kernel leaves it for every query row (the pass runs right after a FlashAttention
+     * prefill, Sec. 4.1, which keeps this value per row).  When given, the scores are computed in
+     * ONE sweep over K: A = exp(logit - row_lse) needs no normalising sweep of its own.  The values
+     * are trusted: a row_lse that is not the normaliser of the q_win and k passed in scales that
+     * row's attention weights by exp(true - given).  The values of sequences that are returned
+     * unchanged are ignored. */
+    const float *row_lse;
+    int reserved[6];
 } sablock_params_t;
 
 void sablock_params_default(sablock_params_t *p);

@@ -39,7 +39,7 @@ class Params(C.Structure):
         ("alpha", C.c_float), ("eta", C.c_float), ("eps", C.c_float), ("tau", C.c_float),
         ("pool_kernel", C.c_int), ("pool_mode", C.c_int), ("budget_includes_window", C.c_int),
         ("delim_bitmap", C.c_void_p), ("vocab_size", C.c_int),
-        ("score_impl", C.c_int), ("l2_lag_tiles", C.c_int), ("reserved", C.c_int * 7),
+        ("score_impl", C.c_int), ("reserved0", C.c_int), ("row_lse", C.c_void_p), ("reserved", C.c_int * 6),
     ]
 
 
@@ -118,6 +118,11 @@ def make_params(n_q_heads: int, n_kv_heads: int, head_dim: int, window: int, dty
     for k, v in kw.items():
         if not hasattr(p, k):
             raise AttributeError(k)
+        if k == "row_lse" and isinstance(v, torch.Tensor):
+            if v.dtype != torch.float32 or not v.is_contiguous():
+                raise TypeError("row_lse must be a contiguous float32 tensor")
+            p._row_lse_ref = v                # keep the device buffer alive as long as the block
+            v = v.data_ptr()
         setattr(p, k, v)
     return p
 

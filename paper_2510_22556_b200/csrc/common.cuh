@@ -112,17 +112,6 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
-// Optional counters of the polls of the bounded waits (compiled in with -DSABLOCK_TRACE).
-#ifdef SABLOCK_TRACE
-__device__ unsigned long long g_spin[8];
-#define SPIN_COUNT(i, n)                                                                      \
-    do {                                                                                      \
-        if ((threadIdx.x & 31) == 0 && (n) > 0) atomicAdd(&g_spin[i], (unsigned long long)(n)); \
-    } while (0)
-#else
-#define SPIN_COUNT(i, n) do { } while (0)
-#endif
-
 // Non-blocking probes of two barriers whose latencies overlap (both tests are issued before
 // either result is used).
 __device__ __forceinline__ void mbar_test_wait2(uint32_t bar_a, uint32_t parity_a, uint32_t bar_b, uint32_t parity_b,
@@ -152,13 +141,8 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     int spins = 0;
     while (true) {
         if (mbar_try_wait(bar, parity)) {
-            SPIN_COUNT(0, spins + 1);
-            SPIN_COUNT(5, 1);
             return true;
         }
-#ifdef SABLOCK_WAIT_SLEEP_NS
-        __nanosleep(SABLOCK_WAIT_SLEEP_NS);
-#endif
         if ((++spins & 3) == 0) {
             if (*abort_flag) return false;
             if (clock64() - t0 > kWaitLimitCycles) {
@@ -213,6 +197,15 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* m, 
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3),
         "l"(policy)
         : "memory");
+}
+
+// Untiled bulk copy global -> this CTA's shared memory; both addresses 16-byte aligned, `bytes` a
+// multiple of 16; completion is signalled on `bar` by bytes.
+__device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
 }
 
 // --- tensor memory and tcgen05 -----------------------------------------------------------

@@ -64,8 +64,8 @@ struct Plan {
     int keep_words, long_cap, seg_tiles;
     // workspace offsets
     size_t o_status, o_ticket, o_long_count, o_tile_state, o_keep, o_arrive, o_done, o_top, control_bytes;
-    size_t o_seg_id, o_seg_start, o_n_seg, o_s_raw, o_s, o_e, o_sr, o_part, o_lse, o_thr, o_cut, o_long_list,
-        o_phi, o_rank, o_fpart, total;
+    size_t o_seg_id, o_seg_start, o_n_seg, o_s_raw, o_s, o_e, o_sr, o_part, o_lse, o_neg_lse, o_thr, o_cut, o_long_list,
+        o_phi, o_fpart, total;
 };
 
 bool tc_eligible(const sablock_params_t* p)
@@ -105,6 +105,23 @@ int fused_cta_limit()
         have[dev] = true;
     }
     return cached[dev];
+}
+
+// SMs of the current device; 148, a B200's count, where no device can be asked (sizing a
+// workspace on a host without a GPU).  The tiles per CTA of the two-launch score kernels, and with
+// them the size of their partial-sum scratch, follow from it: size a workspace with the device
+// current that will use it.
+int sm_count()
+{
+    static int cached[64];
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return 148; }
+    if (cached[dev] > 0) return cached[dev];
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) {
+        cudaGetLastError();
+        return 148;
+    }
+    return cached[dev] = sms;
 }
 
 sablock_status_t validate_params(const sablock_params_t* p)
@@ -177,8 +194,9 @@ sablock_status_t make_plan(const sablock_params_t* p, int n_layers, int n_seqs, 
     pl->use_fused = pl->use_tc && p->score_impl != SABLOCK_SCORE_TENSOR && fused_eligible(p);
     if (pl->use_tc) {
         long long work1 = tiles * g.Hkv * pl->n_prob, work2 = tiles * pl->n_prob;
-        pl->tpc1 = (int)fmin(8.0, fmax(1.0, (double)(work1 / (148 * 4))));
-        pl->tpc2 = (int)fmin(4.0, fmax(1.0, (double)(work2 / (148 * 4))));
+        const int sms = sm_count();
+        pl->tpc1 = (int)fmin(8.0, fmax(1.0, (double)(work1 / (sms * 4))));
+        pl->tpc2 = (int)fmin(4.0, fmax(1.0, (double)(work2 / (sms * 4))));
         pl->n_chunks = (int)((tiles + pl->tpc1 - 1) / pl->tpc1);
     } else {
         pl->tpc1 = pl->tpc2 = 1;
@@ -211,11 +229,11 @@ sablock_status_t make_plan(const sablock_params_t* p, int n_layers, int n_seqs, 
                                      : (size_t)pl->n_prob * g.H * g.window * pl->n_chunks;
     pl->o_part = take(sizeof(float2) * part_n);
     pl->o_lse = take(sizeof(float) * (size_t)pl->n_prob * g.H * g.window);
+    pl->o_neg_lse = take(sizeof(float) * (size_t)pl->n_prob * g.H * g.window);
     pl->o_thr = take(sizeof(unsigned) * pl->n_prob);
     pl->o_cut = take(sizeof(int) * pl->n_prob);
     pl->o_long_list = take(sizeof(int) * (size_t)pl->n_prob * pl->long_cap);
     pl->o_phi = take(sizeof(double) * ntok);
-    pl->o_rank = take(sizeof(int) * ntok);
     pl->o_fpart = take(pl->use_fused ? sizeof(float2) * (size_t)kFuMaxCtas * kFuPartSlots * 128 : 0);
     pl->total = o;
     return SABLOCK_OK;
@@ -349,6 +367,16 @@ sablock_status_t run_score(const Plan& pl, const sablock_params_t* p, const void
     sb.n_chunks = pl.n_chunks;
     int* status = at<int>(ws, pl.o_status);
     const Strides ks = k_strides(p, g.total_tokens);
+    // Single-sweep mode (Sec. 4.1: the pass follows a prefill whose attention kernel keeps the
+    // log of Eq. 2's normaliser per query row): no pass over K for the row statistics.
+    const bool have_lse = p->row_lse != nullptr;
+    float* neg_lse2 = at<float>(ws, pl.o_neg_lse);
+    if (have_lse) {
+        if (reinterpret_cast<uintptr_t>(p->row_lse) & 3) return SABLOCK_ERR_INVALID_ARG;
+        const size_t n = (size_t)pl.n_prob * g.H * g.window;
+        lse_import_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(p->row_lse, sb.lse2, neg_lse2, n);
+        SAB_TRY(check_launch());
+    }
     if (pl.use_tc) {
         CUtensorMap tmQ, tmK;
         SAB_TRY(make_tensor_maps(pl, p, q, k, &tmQ, &tmK));
@@ -366,6 +394,7 @@ sablock_status_t run_score(const Plan& pl, const sablock_params_t* p, const void
             fa.c2 = c2; fa.eps = p->eps;
             fa.part = at<float2>(ws, pl.o_fpart);
             fa.lse2 = sb.lse2;
+            fa.neg_lse2 = have_lse ? neg_lse2 : nullptr;
             fa.arrive = at<int>(ws, pl.o_arrive);
             fa.done = at<int>(ws, pl.o_done);
             fa.s_out = s; fa.e_out = e; fa.status = status;
@@ -390,11 +419,15 @@ sablock_status_t run_score(const Plan& pl, const sablock_params_t* p, const void
         if (cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, smem1) != cudaSuccess)
             return SABLOCK_ERR_CUDA;
         dim3 grid1(pl.n_chunks, g.Hkv, pl.n_prob);
-        k1<<<grid1, kTcThreads, smem1, stream>>>(tmQ, tmK, g, c2, sb, pl.tpc1, status);
-        SAB_TRY(check_launch());
+        if (!have_lse) {
+            k1<<<grid1, kTcThreads, smem1, stream>>>(tmQ, tmK, g, c2, sb, pl.tpc1, status);
+            SAB_TRY(check_launch());
+        }
         prof_mark(1, stream);
-        lse_merge_tc<<<dim3(g.Hkv, pl.n_prob), 128, 0, stream>>>(g, sb, pl.tpc1);
-        SAB_TRY(check_launch());
+        if (!have_lse) {
+            lse_merge_tc<<<dim3(g.Hkv, pl.n_prob), 128, 0, stream>>>(g, sb, pl.tpc1);
+            SAB_TRY(check_launch());
+        }
         prof_mark(2, stream);
         switch (g.window) {
             case 8: return launch_p2_tc<8>(pl, tmQ, tmK, c2, p->eps, sb, s, e, status, stream);
@@ -412,12 +445,16 @@ sablock_status_t run_score(const Plan& pl, const sablock_params_t* p, const void
         auto k1 = score_p1_simt<__nv_bfloat16>;
         if (cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, smem1) != cudaSuccess)
             return SABLOCK_ERR_CUDA;
-        k1<<<grid1, kSimtThreads, smem1, stream>>>(g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, ks.tok, ks.head,
-                                                   ks.layer, c2, sb);
-        SAB_TRY(check_launch());
+        if (!have_lse) {
+            k1<<<grid1, kSimtThreads, smem1, stream>>>(g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, ks.tok, ks.head,
+                                                       ks.layer, c2, sb);
+            SAB_TRY(check_launch());
+        }
         prof_mark(1, stream);
-        lse_merge_simt<<<gridm, 128, 0, stream>>>(g, sb);
-        SAB_TRY(check_launch());
+        if (!have_lse) {
+            lse_merge_simt<<<gridm, 128, 0, stream>>>(g, sb);
+            SAB_TRY(check_launch());
+        }
         prof_mark(2, stream);
         score_p2_simt<__nv_bfloat16><<<grid2, kSimtThreads, smem2, stream>>>(
             g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, ks.tok, ks.head, ks.layer, c2, p->eps, sb, s, e);
@@ -425,11 +462,15 @@ sablock_status_t run_score(const Plan& pl, const sablock_params_t* p, const void
         auto k1 = score_p1_simt<float>;
         if (cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, smem1) != cudaSuccess)
             return SABLOCK_ERR_CUDA;
-        k1<<<grid1, kSimtThreads, smem1, stream>>>(g, (const float*)q, (const float*)k, ks.tok, ks.head, ks.layer, c2, sb);
-        SAB_TRY(check_launch());
+        if (!have_lse) {
+            k1<<<grid1, kSimtThreads, smem1, stream>>>(g, (const float*)q, (const float*)k, ks.tok, ks.head, ks.layer, c2, sb);
+            SAB_TRY(check_launch());
+        }
         prof_mark(1, stream);
-        lse_merge_simt<<<gridm, 128, 0, stream>>>(g, sb);
-        SAB_TRY(check_launch());
+        if (!have_lse) {
+            lse_merge_simt<<<gridm, 128, 0, stream>>>(g, sb);
+            SAB_TRY(check_launch());
+        }
         prof_mark(2, stream);
         score_p2_simt<float><<<grid2, kSimtThreads, smem2, stream>>>(g, (const float*)q, (const float*)k, ks.tok,
                                                                      ks.head, ks.layer, c2, p->eps, sb, s, e);
@@ -525,8 +566,8 @@ sablock_status_t run_select(const Plan& pl, const sablock_params_t* p, const flo
     search_kernel<<<dim3(gx, pl.n_prob), kSearchWarps * 32, 0, stream>>>(g, cands, s_ref, seg_start, n_seg, thr, cut,
                                                                         p->tau, so);
     SAB_TRY(check_launch());
-    search_long_kernel<<<dim3(4, pl.n_prob), kLongThreads, 0, stream>>>(g, cands, s_ref, seg_start, thr, cut, p->tau, so,
-                                                                       at<double>(ws, pl.o_phi), at<int>(ws, pl.o_rank));
+    search_long_kernel<<<dim3(8, pl.n_prob), kLongThreads, 0, stream>>>(g, cands, s_ref, seg_start, thr, cut, p->tau, so,
+                                                                       at<double>(ws, pl.o_phi));
     SAB_TRY(check_launch());
     prof_mark(6, stream);
     index_kernel<<<pl.n_prob, kIdxThreads, 0, stream>>>(g, so.keep, pl.keep_words, out_idx, out_n_keep,
@@ -889,13 +930,5 @@ sablock_status_t sablock_compress_layers_host(const sablock_params_t* p, int n_l
         return SABLOCK_ERR_CUDA;
     return cudaStreamSynchronize(st) == cudaSuccess ? SABLOCK_OK : SABLOCK_ERR_CUDA;
 }
-
-#ifdef SABLOCK_TRACE
-/* Trace builds only: copies the cycle stamps of the traced CTAs to host memory. */
-int sablock_trace_dump(long long* out)
-{
-    return (int)cudaMemcpyFromSymbol(out, sab::g_trace, sizeof(sab::g_trace));
-}
-#endif
 
 }  // extern "C"

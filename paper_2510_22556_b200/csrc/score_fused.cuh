@@ -37,63 +37,25 @@ constexpr int kFuThreads = 608;
 constexpr int kFuEpiWarp0 = 2;
 constexpr int kFuEpiWarps = 16;
 constexpr int kFuHelpWarp = 18;
-#ifndef SABLOCK_K_STAGES
-#define SABLOCK_K_STAGES 3
-#endif
-#ifndef SABLOCK_Q_BUFS
-#define SABLOCK_Q_BUFS 3
-#endif
-constexpr int kFuStages = SABLOCK_K_STAGES;   // K tile ring
-constexpr int kFuQBufs = SABLOCK_Q_BUFS;      // query-block buffers: phases n - 1 (sweep B), n (sweep A), n + 1 (loading ahead)
+constexpr int kFuStages = 3;                 // K tile ring
+constexpr int kFuQBufs = 3;                  // query-block buffers: phases n - 1 (sweep B), n (sweep A), n + 1 (loading ahead)
 constexpr int kFuMaxTilesPerCta = 7;         // \bar A slots in tensor memory: 7 x 32 columns
 constexpr int kFuAbarCol0 = 256;             // columns [0, 256): two logit accumulators
 constexpr int kFuTmemCols = 512;
-#ifndef SABLOCK_LEAD
-#define SABLOCK_LEAD 2
-#endif
-constexpr int kFuLead = SABLOCK_LEAD;                   // sweep A runs at least this many tiles ahead of sweep B
-#ifndef SABLOCK_RUN_AHEAD
-#define SABLOCK_RUN_AHEAD 0
-#endif
-constexpr int kFuRunAhead = SABLOCK_RUN_AHEAD;
+constexpr int kFuLead = 2;                   // sweep A runs at least this many tiles ahead of sweep B
 constexpr int kFuPartSlots = 4;              // ring of per-phase partial buffers in global memory
-constexpr int kFuLseSlots = 4;               // ring of log-sum-exp buffers in shared memory
+constexpr int kFuLseSlots = 8;               // ring of log-sum-exp buffers in shared memory
 constexpr int kFuMaxCtasDev = 256;           // upper bound on the CTAs of one launch
 constexpr int kFuTileBytes = 2 * kAtomBytes; // 128 rows x 128 bf16
 constexpr int kFuSmemBytes = 1024 + (kFuQBufs + kFuStages) * kFuTileBytes;
-#ifndef SABLOCK_RELEASE_AT
-#define SABLOCK_RELEASE_AT 0
-#endif
-// When an epilogue set hands its accumulator back to the MMA issuer: 0 = as soon as the logits
-// are in registers, 1 = after half of the step's arithmetic, 2 = when the step is done.  A late
-// release makes the tensor core pace the sets: their products cannot overlap, so the two sets
-// settle half a step apart and one computes while the other waits, loads and fetches its next
-// step, instead of both doing so at the same time.
-constexpr int kReleaseAt = SABLOCK_RELEASE_AT;
-#ifndef SABLOCK_F32X2
-#define SABLOCK_F32X2 1
-#endif
-#ifndef SABLOCK_AHEAD
-#define SABLOCK_AHEAD 1
-#endif
-constexpr bool kAhead = SABLOCK_AHEAD != 0;
-#ifndef SABLOCK_XU_PASS_A
-#define SABLOCK_XU_PASS_A 1      // sweep A passes the turn after this many of its two chunks (1 measured best)
-#endif
-#ifndef SABLOCK_XU_PASS_B
-#define SABLOCK_XU_PASS_B 3      // sweep B passes the turn after this many of its four heads (3 measured best)
-#endif
-#ifndef SABLOCK_XU_TURNS
-#define SABLOCK_XU_TURNS 1
-#endif
 // The two epilogue sets take turns at the exponentials.  The special-function unit is the busiest
 // unit of the kernel; two sets that share it freely end up in lockstep, both computing and then
 // both going through the latencies between two steps (step record, accumulator barrier,
 // tensor-memory loads) with the unit idle.  With turns, set s starts the exponentials of its k-th
 // step only when the other set is well into those of its own preceding step (halfway in sweep A,
 // three heads of four in sweep B), which keeps the sets apart: while one goes through the
-// latencies the other has the unit.
-constexpr bool kXuTurns = SABLOCK_XU_TURNS != 0;
+// latencies the other has the unit.  An epilogue set hands its accumulator back to the MMA issuer
+// as soon as the logits are in registers.
 
 struct FusedArgs {
     int cpp;                 // CTAs per group (one group works on one problem at a time)
@@ -103,37 +65,14 @@ struct FusedArgs {
     float eps;
     float2* part;            // [n_groups][kFuPartSlots][cpp][128] row statistics (m, l)
     float* lse2;             // [n_prob][Hkv * 128] log2-sum-exp2 per window row
+    const float* neg_lse2;   // single-sweep mode: minus the log2-sum-exp2 of every window row, known beforehand
+                             // (same layout as lse2; NULL = two sweeps, the kernel works the normalisers out itself)
     int* arrive;             // [n_prob][Hkv]
     int* done;               // [n_prob][Hkv]
     float* s_out;            // [n_layers][total_tokens]
     float* e_out;
     int* status;
 };
-
-// Optional cycle-stamp trace of a few CTAs (compiled in with -DSABLOCK_TRACE; off otherwise):
-// role 0 = producer, 1 = MMA issuers (per step), 2 / 3 = first thread of epilogue set 0 / 1
-// (per own step), 4 / 5 = hand-over warp per phase (4: row sums taken, published, all CTAs in,
-// merged; 5: merges of all CTAs in, log-sum-exps fetched).
-#ifdef SABLOCK_TRACE
-constexpr int kTraceOps = 600;
-__device__ long long g_trace[4][6][kTraceOps][8];   // [traced CTA][role][step][event]
-#ifdef SABLOCK_TRACE_MIN       // epilogue: only "accumulator released" and "step done", to keep the probes' own cost out
-#define FU_TRACE_KEEP(role, ev) ((role) < 2 || (role) > 3 || (ev) == 2 || (ev) == 3 || (ev) == SABLOCK_TRACE_MIN || (SABLOCK_TRACE_MIN == 67 && ((ev) == 6 || (ev) == 7)))
-#else
-#define FU_TRACE_KEEP(role, ev) true
-#endif
-#define FU_TRACE(role, n, ev)                                                                 \
-    do {                                                                                      \
-        if (FU_TRACE_KEEP(role, ev) && tslot >= 0 && (n) < kTraceOps) g_trace[tslot][role][n][ev] = clock64(); \
-    } while (0)
-#define FU_TRACE_VAL(role, n, ev, val)                                                        \
-    do {                                                                                      \
-        if (tslot >= 0 && (n) < kTraceOps) g_trace[tslot][role][n][ev] = (val);               \
-    } while (0)
-#else
-#define FU_TRACE(role, n, ev) do { } while (0)
-#define FU_TRACE_VAL(role, n, ev, val) do { } while (0)
-#endif
 
 struct FuBarriers {
     uint64_t full[kFuStages];
@@ -235,8 +174,7 @@ struct FuIter {
             op.kind = kOpPairEnd;
             return op;
         }
-        // how far sweep A may run into the phase after next (in tiles) while sweep B waits
-        const bool can_a = a_ph < n_phases && ia < pa.n_a && (a_ph <= b_ph + 1 || ia < kFuRunAhead);
+        const bool can_a = a_ph < n_phases && ia < pa.n_a && a_ph <= b_ph + 1;
         const bool can_b = b_ph < a_ph && ib < q0.n_b;
         if (!can_a && !can_b) { op.kind = kOpStop; return op; }
         const bool lead_needed = a_ph == b_ph + 1 && ia < ib + kFuLead;
@@ -266,8 +204,8 @@ constexpr int kStepQPar = 1 << 11;      // parity of that buffer's load
 constexpr int kStepRelShift = 12;       // bits 12-14: before this step, query-block buffer i has seen its last product
 constexpr int kStepMask = 1 << 15;      // sweep A tile that reaches the causal boundary
 constexpr int kStepNewQ = 1 << 16;      // first step that uses this load of the query block
-constexpr int kStepLseShift = 17;       // (epilogue rings) bits 17-18: log-sum-exp buffer of the phase, bit 19: parity of its fill
-constexpr int kStepStop = 1 << 20;      // (epilogue rings) no further step for this set
+constexpr int kStepLseShift = 17;       // (epilogue rings) bits 17-19: log-sum-exp buffer of the phase, bit 20: parity of its fill
+constexpr int kStepStop = 1 << 21;      // (epilogue rings) no further step for this set
 constexpr int kStepTagShift = 24;       // (epilogue rings) bits 24-31: which use of the ring slot this is (never 0)
 
 constexpr int kFuRing = 16;
@@ -398,7 +336,6 @@ __device__ __forceinline__ bool wait_counter(const int* ctr, int target, volatil
     int spins = 0;
     while (true) {
         if (ld_acquire(ctr) >= target) return true;
-        SPIN_COUNT(3, 1);
         __nanosleep(64);
         if ((++spins & 15) == 0) {
             if (*abort_flag || ld_acquire(status) != 0 || clock64() - t0 > kWaitLimitCycles) {
@@ -410,18 +347,33 @@ __device__ __forceinline__ bool wait_counter(const int* ctr, int target, volatil
 }
 
 
-__device__ __forceinline__ int sched_count(const FuSched& sc)
+// The step rings and the small counters of FuSched are handed between threads of the CTA with
+// release stores and acquire loads (CTA scope): a reader that sees a count, a tag or a counter
+// value also sees every shared-memory store the writer made before publishing it, and its own
+// later loads of the record cannot be served from before that point.
+__device__ __forceinline__ void st_release_cta(const volatile void* p, int v)
+{
+    asm volatile("st.release.cta.shared.s32 [%0], %1;" ::"r"(smem_u32((const void*)p)), "r"(v) : "memory");
+}
+__device__ __forceinline__ int ld_acquire_cta(const volatile void* p)
 {
     int v;
-    asm volatile("ld.volatile.shared.s32 %0, [%1];" : "=r"(v) : "r"(smem_u32((const void*)&sc.count)) : "memory");
+    asm volatile("ld.acquire.cta.shared.s32 %0, [%1];" : "=r"(v) : "r"(smem_u32((const void*)p)) : "memory");
     return v;
 }
+__device__ __forceinline__ int4 ld_shared_v4(uint32_t src)
+{
+    int4 out;
+    asm volatile("ld.volatile.shared.v4.s32 {%0, %1, %2, %3}, [%4];" : "=r"(out.x), "=r"(out.y), "=r"(out.z), "=r"(out.w) : "r"(src) : "memory");
+    return out;
+}
+
+__device__ __forceinline__ int sched_count(const FuSched& sc) { return ld_acquire_cta(&sc.count); }
 __device__ __forceinline__ void sched_post(FuSched& sc, int idx, int4 step)
 {
     const uint32_t dst = smem_u32(&sc.ring[idx % kFuRing]);
     asm volatile("st.volatile.shared.v4.s32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(step.x), "r"(step.y), "r"(step.z), "r"(step.w) : "memory");
-    // shared-memory stores of one thread become visible in order: the counter after the step
-    asm volatile("st.volatile.shared.s32 [%0], %1;" ::"r"(smem_u32((const void*)&sc.count)), "r"(idx + 1) : "memory");
+    st_release_cta(&sc.count, idx + 1);       // the record before the count
 }
 // Waits (bounded) until step `idx` is posted and reads it; false when there is no such step or the
 // wait gave up.
@@ -430,57 +382,31 @@ __device__ __forceinline__ bool sched_get(FuSched& sc, int idx, int4& out, volat
     if (sched_count(sc) <= idx) {
         const long long t0 = clock64();
         while (sched_count(sc) <= idx) {
-            SPIN_COUNT(1, 1);
-            if (sc.final_) {
+            if (ld_acquire_cta(&sc.final_)) {
                 if (sched_count(sc) <= idx) return false;
                 break;
             }
             if (*abort_flag || clock64() - t0 > kWaitLimitCycles) { *abort_flag = 1; return false; }
         }
     }
-    const uint32_t src = smem_u32(&sc.ring[idx % kFuRing]);
-    asm volatile("ld.volatile.shared.v4.s32 {%0, %1, %2, %3}, [%4];" : "=r"(out.x), "=r"(out.y), "=r"(out.z), "=r"(out.w) : "r"(src) : "memory");
+    out = ld_shared_v4(smem_u32(&sc.ring[idx % kFuRing]));
     return true;
 }
 
-// Posts the k-th step of an epilogue set: payload first, then the tagged flags word.
+// Posts the k-th step of an epilogue set: payload first, then the tagged flags word (release).
 __device__ __forceinline__ void sched_post_set(FuSched& sc, int set, int k, int4 step)
 {
     const uint32_t dst = smem_u32(&sc.sring[set][k % kFuSetRing]);
     const int tag = ((k / kFuSetRing) & 0x7f) + 1;
     asm volatile("st.volatile.shared.s32 [%0], %1;" ::"r"(dst + 4), "r"(step.y) : "memory");
     asm volatile("st.volatile.shared.v2.s32 [%0], {%1, %2};" ::"r"(dst + 8), "r"(step.z), "r"(step.w) : "memory");
-    asm volatile("st.volatile.shared.s32 [%0], %1;" ::"r"(dst), "r"(step.x | (tag << kStepTagShift)) : "memory");
+    st_release_cta(&sc.sring[set][k % kFuSetRing], step.x | (tag << kStepTagShift));
 }
-// Reads the k-th step of an epilogue set, waiting (bounded) until it is posted.  The flags word is
-// read before the payload, so a matching tag means the payload is the one posted with it.
-__device__ __forceinline__ bool sched_get_set(FuSched& sc, int set, int k, int4& out, volatile int* abort_flag)
-{
-    const uint32_t src = smem_u32(&sc.sring[set][k % kFuSetRing]);
-    const int tag = ((k / kFuSetRing) & 0x7f) + 1;
-    long long t0 = 0;
-    int spins = 0;
-    while (true) {
-        int fl;
-        asm volatile("ld.volatile.shared.s32 %0, [%1];" : "=r"(fl) : "r"(src) : "memory");
-        asm volatile("ld.volatile.shared.v4.s32 {%0, %1, %2, %3}, [%4];" : "=r"(out.x), "=r"(out.y), "=r"(out.z), "=r"(out.w) : "r"(src) : "memory");
-        if (((unsigned)fl >> kStepTagShift) == (unsigned)tag) {
-            out.x = fl;
-            return true;
-        }
-        if (spins++ == 0) t0 = clock64();
-        SPIN_COUNT(2, 1);
-        if ((spins & 15) == 0 && (*abort_flag || clock64() - t0 > kWaitLimitCycles)) { *abort_flag = 1; return false; }
-    }
-}
-
-// The flags word of the k-th step of an epilogue set as it stands (posted or not), and whether a
-// flags word read that way is the posted k-th step.
+// The flags word of the k-th step of an epilogue set as it stands (posted or not; acquire), and
+// whether a flags word read that way is the posted k-th step.
 __device__ __forceinline__ int sched_peek_flags(FuSched& sc, int set, int k)
 {
-    int fl;
-    asm volatile("ld.volatile.shared.s32 %0, [%1];" : "=r"(fl) : "r"(smem_u32(&sc.sring[set][k % kFuSetRing])) : "memory");
-    return fl;
+    return ld_acquire_cta(&sc.sring[set][k % kFuSetRing]);
 }
 __device__ __forceinline__ bool sched_flags_posted(int fl, int k)
 {
@@ -489,8 +415,24 @@ __device__ __forceinline__ bool sched_flags_posted(int fl, int k)
 // Payload of a step whose flags word has been seen posted.
 __device__ __forceinline__ void sched_payload(FuSched& sc, int set, int k, int4& out)
 {
-    asm volatile("ld.volatile.shared.v4.s32 {%0, %1, %2, %3}, [%4];"
-                 : "=r"(out.x), "=r"(out.y), "=r"(out.z), "=r"(out.w) : "r"(smem_u32(&sc.sring[set][k % kFuSetRing])) : "memory");
+    out = ld_shared_v4(smem_u32(&sc.sring[set][k % kFuSetRing]));
+}
+// Reads the k-th step of an epilogue set, waiting (bounded) until it is posted: the flags word is
+// acquired first, so a matching tag means the payload read after it is the one posted with it.
+__device__ __forceinline__ bool sched_get_set(FuSched& sc, int set, int k, int4& out, volatile int* abort_flag)
+{
+    long long t0 = 0;
+    int spins = 0;
+    while (true) {
+        const int fl = sched_peek_flags(sc, set, k);
+        if (sched_flags_posted(fl, k)) {
+            sched_payload(sc, set, k, out);
+            out.x = fl;
+            return true;
+        }
+        if (spins++ == 0) t0 = clock64();
+        if ((spins & 15) == 0 && (*abort_flag || clock64() - t0 > kWaitLimitCycles)) { *abort_flag = 1; return false; }
+    }
 }
 
 // First wait of the launch that gave up: (code, CTA, warp) goes to the word after the status word.
@@ -560,7 +502,6 @@ __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b)
 // Sum of exp2(v * c2 - m) over 32 logits of one window row.
 __device__ __forceinline__ float chunk_expsum(const uint32_t (&r)[32], float c2, float m)
 {
-#if SABLOCK_F32X2
     const uint64_t cc = pack2(c2, c2), mm = pack2(-m, -m);
     uint64_t s0 = pack2(0.f, 0.f), s1 = s0;
 #pragma unroll
@@ -575,17 +516,6 @@ __device__ __forceinline__ float chunk_expsum(const uint32_t (&r)[32], float c2,
     unpack2(s0, a, b);
     unpack2(s1, c, d);
     return (a + b) + (c + d);
-#else
-    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-#pragma unroll
-    for (int i = 0; i < 32; i += 4) {
-        s0 += ex2_approx(fmaf(__uint_as_float(r[i + 0]), c2, -m));
-        s1 += ex2_approx(fmaf(__uint_as_float(r[i + 1]), c2, -m));
-        s2 += ex2_approx(fmaf(__uint_as_float(r[i + 2]), c2, -m));
-        s3 += ex2_approx(fmaf(__uint_as_float(r[i + 3]), c2, -m));
-    }
-    return (s0 + s1) + (s2 + s3);
-#endif
 }
 __device__ __forceinline__ float chunk_max(const uint32_t (&r)[32])
 {
@@ -638,7 +568,6 @@ struct RowSum {
 __device__ __forceinline__ void accumulate_head16(float (&accw)[16], const uint32_t (&r)[16], const float* lse, float c2)
 {
     const float4* l4 = reinterpret_cast<const float4*>(lse);
-#if SABLOCK_F32X2
     const uint64_t cc = pack2(c2, c2);
 #pragma unroll
     for (int i = 0; i < 16; i += 4) {
@@ -649,17 +578,143 @@ __device__ __forceinline__ void accumulate_head16(float (&accw)[16], const uint3
         unpack2(add2(pack2(accw[i + 0], accw[i + 1]), pack2(ex2_approx(a), ex2_approx(b))), accw[i + 0], accw[i + 1]);
         unpack2(add2(pack2(accw[i + 2], accw[i + 3]), pack2(ex2_approx(c), ex2_approx(d))), accw[i + 2], accw[i + 3]);
     }
-#else
-#pragma unroll
-    for (int i = 0; i < 16; i += 4) {
-        const float4 ls = l4[i >> 2];
-        accw[i + 0] += ex2_approx(fmaf(__uint_as_float(r[i + 0]), c2, ls.x));
-        accw[i + 1] += ex2_approx(fmaf(__uint_as_float(r[i + 1]), c2, ls.y));
-        accw[i + 2] += ex2_approx(fmaf(__uint_as_float(r[i + 2]), c2, ls.z));
-        accw[i + 3] += ex2_approx(fmaf(__uint_as_float(r[i + 3]), c2, ls.w));
-    }
-#endif
 }
+
+// ---- producer of the single-sweep mode ----------------------------------------------------------
+// With the log-sum-exp of every window row known beforehand there is no sweep A and no hand-over
+// between CTAs: the producer walks the phases = (problem, KV head) in which this CTA has token
+// tiles and posts one sweep-B step per tile.  The query block and the 128 log-sum-exps of a phase
+// are fetched one phase ahead: the former into query-block buffer a % 3 (a counts this CTA's
+// phases with tiles), the latter by a bulk copy into log-sum-exp buffer a % 8.  A log-sum-exp
+// buffer is written again eight of this CTA's phases later; the producer is never more than six
+// steps ahead of the oldest step an epilogue set may still be working on (three K stages, two
+// accumulators, the epilogue hands an accumulator back before it is done with the step), and a
+// phase has at least one step, so that buffer has been read for the last time by then.
+struct FuSinglePhase {
+    int phase, prob, j, layer, tok_base, Tn, n_b;
+};
+
+__device__ __forceinline__ void fu_single_advance(FuSinglePhase& c, const Geo& g, int group, int n_groups, int rank, int cpp,
+                                                  int n_phases)
+{
+    while (true) {
+        ++c.phase;
+        if (c.phase >= n_phases) { c.phase = n_phases; return; }
+        if (c.j >= 0 && c.j + 1 < g.Hkv) {             // same problem, next KV head
+            ++c.j;
+        } else {                                       // next problem of the group: the divisions are paid here
+            c.prob = c.j < 0 ? group : c.prob + n_groups;
+            c.j = 0;
+            c.layer = c.prob / g.n_seqs;
+            const int seq = c.prob - c.layer * g.n_seqs;
+            c.tok_base = g.cu[seq];
+            const int L = g.cu[seq + 1] - c.tok_base;
+            c.Tn = L - g.window;
+            const int nt = (c.Tn + kTcTile - 1) / kTcTile;
+            c.n_b = (L > g.n_out && rank < nt) ? (nt - rank + cpp - 1) / cpp : 0;    // else: returned unchanged, or no tile here
+        }
+        if (c.n_b > 0) return;
+    }
+}
+
+__device__ __forceinline__ void fu_produce_single(const CUtensorMap* tmQ, const CUtensorMap* tmK, const Geo& g,
+                                                  const FusedArgs& fa, FuBarriers& sh, FuSched& sched, uint32_t q_smem,
+                                                  uint32_t k_smem, uint32_t lse_smem, volatile int* abort_flag)
+{
+    constexpr int R = 128;
+    const uint64_t pol_k = l2_policy_evict_first();        // every K tile is read once
+    const uint64_t pol_q = l2_policy_evict_last();
+    const int group = blockIdx.x / fa.cpp, rank = blockIdx.x % fa.cpp;
+    const int my_probs = group < fa.n_groups ? (fa.n_prob - group + fa.n_groups - 1) / fa.n_groups : 0;
+    const int n_phases = my_probs * g.Hkv;
+    FuSinglePhase cur;
+    cur.phase = -1; cur.prob = 0; cur.j = -1; cur.layer = 0; cur.tok_base = 0; cur.Tn = 0; cur.n_b = 0;
+    fu_single_advance(cur, g, group, fa.n_groups, rank, fa.cpp, n_phases);
+    FuSinglePhase nxt = cur;
+    if (cur.phase < n_phases) fu_single_advance(nxt, g, group, fa.n_groups, rank, fa.cpp, n_phases);
+
+    // Loads of this CTA's a-th phase with tiles: query block and log-sum-exps.  The buffers must be free.
+    auto issue_phase_loads = [&](const FuSinglePhase& ph, int qb, int ls) {
+        mbar_expect_tx(smem_u32(&sh.qfull[qb]), kFuTileBytes);
+        for (int a = 0; a < 2; ++a)
+            tma_load_2d(q_smem + qb * kFuTileBytes + a * kAtomBytes, tmQ, smem_u32(&sh.qfull[qb]), a * 64,
+                        ph.prob * g.H * g.window + ph.j * R, pol_q);
+        mbar_expect_tx(smem_u32(&sh.lse_full[ls]), R * (uint32_t)sizeof(float));
+        bulk_load_1d(lse_smem + ls * R * (uint32_t)sizeof(float), fa.neg_lse2 + (size_t)ph.prob * g.H * g.window + ph.j * R,
+                     R * (uint32_t)sizeof(float), smem_u32(&sh.lse_full[ls]));
+    };
+
+    int n_steps = 0, pending_rel = 0;
+    int a_idx = 0, qb = 0, ls = 0;                        // this phase: its count, query-block buffer, log-sum-exp buffer
+    unsigned q_uses = 0;                                   // per query-block buffer: parity of the number of loads so far
+    unsigned ls_par = 0;                                   // parity of a_idx / kFuLseSlots
+    int sb0 = -1, sb1 = -1;                                // last phase in which set 0 / set 1 had a step
+    bool ok = true;
+    if (cur.phase < n_phases) {
+        issue_phase_loads(cur, 0, 0);
+        q_uses ^= 1u;
+    }
+    while (ok && cur.phase < n_phases) {
+        const int qb_n = qb == kFuQBufs - 1 ? 0 : qb + 1, ls_n = (ls + 1) & (kFuLseSlots - 1);
+        const bool have_next = nxt.phase < n_phases;
+        bool next_loaded = !have_next;
+        const int qpar = ((q_uses >> qb) & 1u) ^ 1u;       // parity of the load this phase uses (q_uses already counts it)
+        for (int k = 0; k < cur.n_b; ++k) {
+            // the next phase's loads, as soon as its query-block buffer is free (probe only; the
+            // blocking wait comes after the last step of this phase)
+            if (!next_loaded) {
+                const bool fresh = a_idx + 1 < kFuQBufs;
+                if (fresh || mbar_test_wait(smem_u32(&sh.qempty[qb_n]), ((q_uses >> qb_n) & 1u) ^ 1u)) {
+                    issue_phase_loads(nxt, qb_n, ls_n);
+                    q_uses ^= 1u << qb_n;
+                    next_loaded = true;
+                }
+            }
+            int flags = pending_rel | kStepB | (k << kStepKShift) | (qb << kStepQBufShift);
+            pending_rel = 0;
+            if (cur.j == 0) flags |= kStepHead0;
+            if (cur.j == g.Hkv - 1) flags |= kStepHeadLast;
+            if (k == 0) flags |= kStepNewQ;
+            if (qpar) flags |= kStepQPar;
+            const int tok0 = (rank + k * fa.cpp) * kTcTile;
+            const int4 rec = make_int4(flags, tok0, cur.Tn, cur.layer * g.total_tokens + cur.tok_base);
+            sched_post(sched, n_steps, rec);
+            {
+                const int eset = n_steps & 1;
+                int ef = (flags & ~(7 << kStepRelShift)) | ((ls | ((int)ls_par << 3)) << kStepLseShift);
+                if ((eset ? sb1 : sb0) != a_idx) {
+                    if (eset) sb1 = a_idx; else sb0 = a_idx;
+                    ef |= kStepLseWait;
+                }
+                sched_post_set(sched, eset, n_steps >> 1, make_int4(ef, rec.y, rec.z, rec.w));
+            }
+            const int st = n_steps % kFuStages, par = (n_steps / kFuStages) & 1;
+            if (!FU_WAIT(2, mbar_wait(smem_u32(&sh.empty[st]), par ^ 1, abort_flag))) { ok = false; break; }
+            mbar_expect_tx(smem_u32(&sh.full[st]), kFuTileBytes);
+            for (int a = 0; a < 2; ++a)
+                tma_load_4d(k_smem + st * kFuTileBytes + a * kAtomBytes, tmK, smem_u32(&sh.full[st]), a * 64, cur.j,
+                            cur.tok_base + tok0, cur.layer, pol_k);
+            ++n_steps;
+        }
+        if (!ok) break;
+        if (!next_loaded) {
+            if (!FU_WAIT(1, mbar_wait(smem_u32(&sh.qempty[qb_n]), ((q_uses >> qb_n) & 1u) ^ 1u, abort_flag))) break;
+            issue_phase_loads(nxt, qb_n, ls_n);
+            q_uses ^= 1u << qb_n;
+        }
+        pending_rel = 1 << (kStepRelShift + qb);           // this phase's query block has seen its last product
+        cur = nxt;
+        if (have_next) fu_single_advance(nxt, g, group, fa.n_groups, rank, fa.cpp, n_phases);
+        ++a_idx;
+        qb = qb_n;
+        ls = ls_n;
+        if (ls == 0) ls_par ^= 1u;
+    }
+    st_release_cta(&sched.final_, 1);
+    for (int es = 0; es < 2; ++es)
+        sched_post_set(sched, es, (n_steps + 1 - es) >> 1, make_int4(kStepStop, 0, 0, 0));
+}
+
 
 __global__ void __launch_bounds__(kFuThreads, 1)
 score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const Geo g,
@@ -712,15 +767,15 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     const uint32_t tmem = sh.tmem_base;
     volatile int* abort_flag = &sh.abort_flag;
     constexpr int R = 128;                           // window rows per KV head
-#ifdef SABLOCK_TRACE
-    const int tslot = blockIdx.x == 0 ? 0 : blockIdx.x == 5 ? 1 : blockIdx.x == 77 ? 2 : blockIdx.x == gridDim.x - 1 ? 3 : -1;
-#endif
 
     if (warp == 0) {
         // ------------------------------------------------------------------ scheduler + TMA producer
         if (lane == 0) {
             tma_prefetch_desc(&tmQ);
             tma_prefetch_desc(&tmK);
+            if (fa.neg_lse2 != nullptr) {
+                fu_produce_single(&tmQ, &tmK, g, fa, sh, sched, q_smem, k_smem, smem_u32(&lse_s[0][0]), abort_flag);
+            } else {
             const uint64_t pol_a = l2_policy_evict_last();     // first read: keep for sweep B
             const uint64_t pol_b = l2_policy_evict_first();    // second read: last use
             const uint64_t pol_q = l2_policy_evict_last();
@@ -744,7 +799,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     b_counted = it.b_ph;
                     ++b_idx;
                 }
-                const FuOp op = it.next(sched.lse_fetched > b_idx);
+                const FuOp op = it.next(ld_acquire_cta(&sched.lse_fetched) > b_idx);
                 if (op.kind == kOpStop) break;
                 if (op.kind == kOpPairEnd) {
                     // the query block of a phase whose sweep B ended has seen its last product
@@ -779,7 +834,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     int ef = flags & ~(7 << kStepRelShift);
                     if (prev_last_a) ef |= kStepPrevLastA;
                     if (is_b) {
-                        ef |= ((b_idx % kFuLseSlots) | (((b_idx / kFuLseSlots) & 1) << 2)) << kStepLseShift;
+                        ef |= ((b_idx % kFuLseSlots) | (((b_idx / kFuLseSlots) & 1) << 3)) << kStepLseShift;
                         if ((eset ? sb1 : sb0) != b_idx) {
                             if (eset) sb1 = b_idx; else sb0 = b_idx;
                             ef |= kStepLseWait;
@@ -788,7 +843,6 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     sched_post_set(sched, eset, n_steps >> 1, make_int4(ef, rec.y, rec.z, rec.w));
                     prev_last_a = !is_b && op.last;
                 }
-                FU_TRACE(0, n_steps, 3);
                 // ---- query blocks: this step's must be on its way (blocking); the next phase's is
                 // started if its buffer is free (probe only)
                 while (ql_phase < it.n_phases && ql_phase <= op.phase + 1) {
@@ -822,23 +876,21 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 if (!ok) break;
                 // ---- the K tile of the step
                 const int st = n_steps % kFuStages, par = (n_steps / kFuStages) & 1;
-                FU_TRACE(0, n_steps, 0);
                 if (!FU_WAIT(2, mbar_wait(smem_u32(&sh.empty[st]), par ^ 1, abort_flag))) break;
-                FU_TRACE(0, n_steps, 1);
                 mbar_expect_tx(smem_u32(&sh.full[st]), kFuTileBytes);
                 for (int a = 0; a < 2; ++a)
                     tma_load_4d(k_smem + st * kFuTileBytes + a * kAtomBytes, &tmK, smem_u32(&sh.full[st]), a * 64, ph.j,
                                 ph.tok_base + tok0, ph.layer, is_b ? pol_b : pol_a);
-                FU_TRACE(0, n_steps, 2);
                 ++n_steps;
             }
-            sched.final_ = 1;
+            st_release_cta(&sched.final_, 1);
             // the end of each epilogue set's list (also after a wait that gave up: the sets then
             // leave through the abort flag)
             for (int es = 0; es < 2; ++es) {
                 const int k = (n_steps + 1 - es) >> 1;         // steps set es has had
                 const bool other_was_last = prev_last_a && ((n_steps - 1) & 1) != es;
                 sched_post_set(sched, es, k, make_int4(kStepStop | (other_was_last ? kStepPrevLastA : 0), 0, 0, 0));
+            }
             }
         }
     } else if (warp == 1) {
@@ -876,7 +928,6 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 const uint32_t acc = (uint32_t)n & 1u;             // accumulator of the step
                 const uint32_t te_par = (((uint32_t)n >> 1) & 1u) ^ 1u;
                 const uint32_t bar_te = bar_tempty0 + acc * 8u, bar_k = bar_full0 + st * 8u;
-                FU_TRACE(1, n, 0);
                 // both barriers are probed before either result is looked at, so that their
                 // latencies overlap; only a barrier that is not complete yet is waited for
                 bool te_ok, k_ok;
@@ -884,28 +935,23 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 // the first product that uses a load of the query block waits for it
                 if ((flags & kStepNewQ) && !FU_WAIT(3, mbar_wait(smem_u32(&sh.qfull[b]), (flags & kStepQPar) ? 1u : 0u, abort_flag))) break;
                 if (!te_ok && !FU_WAIT(4, mbar_wait(bar_te, te_par, abort_flag))) break;
-                FU_TRACE(1, n, 4);
-                FU_TRACE_VAL(1, n, 5, flags);
                 if (!k_ok && !FU_WAIT(5, mbar_wait(bar_k, kpar, abort_flag))) break;
-                FU_TRACE(1, n, 1);
                 tc_fence_after();
                 // the next step's flags, if it is posted, come in while the products are issued
                 if (sched_count(sched) > n + 1) {
-                    asm volatile("ld.volatile.shared.s32 %0, [%1];" : "=r"(flags_next) : "r"(smem_u32(&sched.ring[(n + 1) % kFuRing])) : "memory");
+                    flags_next = ld_shared_v4(smem_u32(&sched.ring[(n + 1) % kFuRing])).x;
                     have_next = true;
                 }
                 const uint32_t k_lo = k_lo0 + st * kTileLo, q_lo = q_lo0 + b * kTileLo;
                 const bool is_b = (flags & kStepB) != 0;
                 fu_issue_tile(tmem + acc * 128u, is_b ? k_lo : q_lo, is_b ? q_lo : k_lo);   // rows = tokens (B) or window rows (A)
-                FU_TRACE(1, n, 2);
                 tc_commit(bar_empty0 + st * 8u);
                 tc_commit(bar_tfull0 + acc * 8u);
-                FU_TRACE(1, n, 3);
                 ++n;
                 if (++st == kFuStages) { st = 0; kpar ^= 1u; }
             }
         }
-    } else if (warp == kFuHelpWarp) {
+    } else if (warp == kFuHelpWarp && fa.neg_lse2 == nullptr) {
         // ------------------------------------------------------------------ hand-over between CTAs
         // Per phase, in this order: publish this CTA's row sums (the epilogue left the four (set, half)
         // partial sums of every window row in shared memory), merge the sums of all CTAs for this
@@ -933,7 +979,6 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 if (!ok) break;
                 const int buf = n_pub & 1;
                 if (!FU_WAIT(6, mbar_wait(smem_u32(&sh.pub_full[buf]), (uint32_t)((n_pub >> 1) & 1), abort_flag))) break;
-                if (lane == 0) FU_TRACE(4, phase, 0);
                 float2* dst = fa.part + (((size_t)group * kFuPartSlots + (phase % kFuPartSlots)) * fa.cpp + rank) * R;
                 // all partial sums of this lane's four rows first (the loads overlap), then the merges;
                 // the reference exponents are integers, so the rescaling is exact
@@ -958,16 +1003,14 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 __syncwarp();
                 ++n_pub;
                 if (lane == 0) {
-                    sched.pub_done = n_pub;
+                    st_release_cta(&sched.pub_done, n_pub);
                     atomicAdd(fa.arrive + prob * g.Hkv + j, 1);
-                    FU_TRACE(4, phase, 1);
                 }
             }
             if (rank < R) {
                 if (lane == 0) ok = FU_WAIT(12, wait_counter(fa.arrive + prob * g.Hkv + j, n_src, abort_flag, fa.status));
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
-                if (lane == 0) FU_TRACE(4, phase, 2);
                 const float2* pp = fa.part + ((size_t)group * kFuPartSlots + (phase % kFuPartSlots)) * fa.cpp * R;
                 for (int row = rank; row < R; row += fa.cpp) {
                     // one partial per source CTA, merged in index order; all loads of a lane are issued
@@ -1006,7 +1049,6 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 if (lane == 0) {
                     __threadfence();
                     atomicAdd(fa.done + prob * g.Hkv + j, 1);
-                    FU_TRACE(4, phase, 3);
                 }
             }
             // the finished log-sum-exps, if this CTA runs sweep B for the phase
@@ -1014,7 +1056,6 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 if (lane == 0) ok = FU_WAIT(13, wait_counter(fa.done + prob * g.Hkv + j, n_mergers, abort_flag, fa.status));
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
-                if (lane == 0) FU_TRACE(5, phase, 0);
                 const int slot = n_fetch % kFuLseSlots;
                 const float* src = fa.lse2 + (size_t)prob * g.H * g.window + j * R;
 #pragma unroll
@@ -1023,8 +1064,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 ++n_fetch;
                 if (lane == 0) {
                     mbar_arrive(smem_u32(&sh.lse_full[slot]));
-                    sched.lse_fetched = n_fetch;
-                    FU_TRACE(5, phase, 1);
+                    st_release_cta(&sched.lse_fetched, n_fetch);
                 }
             }
         }
@@ -1035,8 +1075,6 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         const int set = (ew >> 2) & 1;
         const int half = ew >> 3;
         const int row = q4 * 32 + lane;                // TMEM lane: window row (sweep A) or token (sweep B)
-        const bool first_thread = (ew & 11) == 0 && lane == 0;       // for the trace
-        (void)first_thread;
         const uint32_t lane_addr = tmem + ((uint32_t)(q4 * 32) << 16);
         const uint32_t acc_addr = lane_addr + (uint32_t)set * 128u;
         const float c2 = fa.c2;
@@ -1048,10 +1086,9 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         // two phases behind).
         auto publish = [&]() -> bool {
             const int buf = n_pub & 1;
-            if (n_pub >= 2 && sched.pub_done < n_pub - 1) {
+            if (n_pub >= 2 && ld_acquire_cta(&sched.pub_done) < n_pub - 1) {
                 const long long t0 = clock64();
-                while (sched.pub_done < n_pub - 1) {
-                    SPIN_COUNT(4, 1);
+                while (ld_acquire_cta(&sched.pub_done) < n_pub - 1) {
                     if (*abort_flag || clock64() - t0 > kWaitLimitCycles) { note_giveup(fa.status, 21); *abort_flag = 1; break; }
                 }
                 if (*abort_flag) return false;
@@ -1068,7 +1105,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         int ahead_flags = 0;
         bool ahead_tfull = false, have_payload = true;
         while (true) {
-            if (kAhead && sched_flags_posted(ahead_flags, n_mine)) {
+            if (sched_flags_posted(ahead_flags, n_mine)) {
                 e.x = ahead_flags;
                 have_payload = false;
             } else {
@@ -1077,24 +1114,19 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 ahead_tfull = false;
             }
             const int flags = e.x;
-            if (first_thread) FU_TRACE(2 + set, n_mine, 5);
-            if (first_thread) FU_TRACE_VAL(2 + set, n_mine, 4, flags);
             // the other set took the last sweep A step of a phase: this thread's row sums are due too
             if ((flags & kStepPrevLastA) && !publish()) break;
             if (flags & kStepStop) break;
             if (!(flags & kStepB)) {
                 {
-                    if (first_thread) FU_TRACE(2 + set, n_mine, 0);
                     if (!ahead_tfull && !FU_WAIT(7, mbar_wait(smem_u32(&sh.tfull[set]), (uint32_t)(n_mine & 1), abort_flag))) break;
-                    if (first_thread) FU_TRACE(2 + set, n_mine, 1);
                     tc_fence_after();
                     uint32_t r0[32], r1[32];
                     tmem_ld32_issue(acc_addr + half * 64, r0);
                     tmem_ld32_issue(acc_addr + half * 64 + 32, r1);
                     tmem_ld_wait();
                     tc_fence_before();
-                    if (kReleaseAt == 0) mbar_arrive(smem_u32(&sh.tempty[set]));   // logits are in registers
-                    if (first_thread) FU_TRACE(2 + set, n_mine, 2);
+                    mbar_arrive(smem_u32(&sh.tempty[set]));   // logits are in registers
                     if (flags & kStepMask) {
                         if (!have_payload) sched_payload(sched, set, n_mine, e);
                         const int tok0 = e.y + half * 64;
@@ -1102,31 +1134,23 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         chunk_mask(r0, tok0, lim);
                         chunk_mask(r1, tok0 + 32, lim);
                     }
-                    if (kXuTurns && !FU_WAIT(9, mbar_wait(smem_u32(&sh.xu[set]), (uint32_t)((n_mine & 1) ^ (set ^ 1)), abort_flag))) break;
-                    if (first_thread) FU_TRACE(2 + set, n_mine, 6);
+                    if (!FU_WAIT(9, mbar_wait(smem_u32(&sh.xu[set]), (uint32_t)((n_mine & 1) ^ (set ^ 1)), abort_flag))) break;
                     rs.add(r0, c2);
-                    if (kXuTurns && SABLOCK_XU_PASS_A == 1) mbar_arrive(smem_u32(&sh.xu[set ^ 1]));
-                    if (kReleaseAt == 1) mbar_arrive(smem_u32(&sh.tempty[set]));
-                    if (kAhead) ahead_flags = sched_peek_flags(sched, set, n_mine + 1);
+                    mbar_arrive(smem_u32(&sh.xu[set ^ 1]));
+                    ahead_flags = sched_peek_flags(sched, set, n_mine + 1);
                     rs.add(r1, c2);
-                    if (kXuTurns && SABLOCK_XU_PASS_A == 2) mbar_arrive(smem_u32(&sh.xu[set ^ 1]));
-                    if (kAhead) ahead_tfull = mbar_test_wait(smem_u32(&sh.tfull[set]), (uint32_t)((n_mine + 1) & 1));
-                    if (kReleaseAt == 2) mbar_arrive(smem_u32(&sh.tempty[set]));
-                    if (first_thread) FU_TRACE(2 + set, n_mine, 7);
-                    if (first_thread) FU_TRACE(2 + set, n_mine, 3);
+                    ahead_tfull = mbar_test_wait(smem_u32(&sh.tfull[set]), (uint32_t)((n_mine + 1) & 1));
                     ++n_mine;
                 }
                 if ((flags & kStepLastA) && !publish()) break;
             } else {
                 {
-                    const int lse_slot = (flags >> kStepLseShift) & 3;
+                    const int lse_slot = (flags >> kStepLseShift) & 7;
                     if (flags & kStepLseWait) {                    // log-sum-exps of this phase (fetched by warp 18)
-                        if (!FU_WAIT(8, mbar_wait(smem_u32(&sh.lse_full[lse_slot]), (uint32_t)((flags >> (kStepLseShift + 2)) & 1), abort_flag)))
+                        if (!FU_WAIT(8, mbar_wait(smem_u32(&sh.lse_full[lse_slot]), (uint32_t)((flags >> (kStepLseShift + 3)) & 1), abort_flag)))
                             break;
                     }
-                    if (first_thread) FU_TRACE(2 + set, n_mine, 0);
                     if (!ahead_tfull && !FU_WAIT(7, mbar_wait(smem_u32(&sh.tfull[set]), (uint32_t)(n_mine & 1), abort_flag))) break;
-                    if (first_thread) FU_TRACE(2 + set, n_mine, 1);
                     tc_fence_after();
                     const float* lj = lse_s[lse_slot] + half * 16;
                     float accw[16];
@@ -1139,23 +1163,15 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     tmem_ld16_issue(acc_addr + 96 + half * 16, v3);
                     tmem_ld_wait();
                     tc_fence_before();
-                    if (kReleaseAt == 0) mbar_arrive(smem_u32(&sh.tempty[set]));
-                    if (first_thread) FU_TRACE(2 + set, n_mine, 2);
-                    if (kXuTurns && !FU_WAIT(9, mbar_wait(smem_u32(&sh.xu[set]), (uint32_t)((n_mine & 1) ^ (set ^ 1)), abort_flag))) break;
-                    if (first_thread) FU_TRACE(2 + set, n_mine, 6);
+                    mbar_arrive(smem_u32(&sh.tempty[set]));
+                    if (!FU_WAIT(9, mbar_wait(smem_u32(&sh.xu[set]), (uint32_t)((n_mine & 1) ^ (set ^ 1)), abort_flag))) break;
                     accumulate_head16(accw, v0, lj, c2);
-                    if (kXuTurns && SABLOCK_XU_PASS_B == 1) mbar_arrive(smem_u32(&sh.xu[set ^ 1]));
                     accumulate_head16(accw, v1, lj + 32, c2);
-                    if (kXuTurns && SABLOCK_XU_PASS_B == 2) mbar_arrive(smem_u32(&sh.xu[set ^ 1]));
-                    if (kReleaseAt == 1) mbar_arrive(smem_u32(&sh.tempty[set]));
-                    if (kAhead) ahead_flags = sched_peek_flags(sched, set, n_mine + 1);
+                    ahead_flags = sched_peek_flags(sched, set, n_mine + 1);
                     accumulate_head16(accw, v2, lj + 64, c2);
-                    if (kXuTurns && SABLOCK_XU_PASS_B == 3) mbar_arrive(smem_u32(&sh.xu[set ^ 1]));
+                    mbar_arrive(smem_u32(&sh.xu[set ^ 1]));
                     accumulate_head16(accw, v3, lj + 96, c2);
-                    if (kXuTurns && SABLOCK_XU_PASS_B == 4) mbar_arrive(smem_u32(&sh.xu[set ^ 1]));
-                    if (kAhead) ahead_tfull = mbar_test_wait(smem_u32(&sh.tfull[set]), (uint32_t)((n_mine + 1) & 1));
-                    if (kReleaseAt == 2) mbar_arrive(smem_u32(&sh.tempty[set]));
-                    if (first_thread) FU_TRACE(2 + set, n_mine, 7);
+                    ahead_tfull = mbar_test_wait(smem_u32(&sh.tfull[set]), (uint32_t)((n_mine + 1) & 1));
                     // \bar A of this token tile, summed over the KV heads seen so far
                     const uint32_t abar_addr = lane_addr + (uint32_t)(kFuAbarCol0 + ((flags >> kStepKShift) & 7) * 32 + half * 16);
                     if (!(flags & kStepHead0)) {
@@ -1197,7 +1213,6 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                             fa.e_out[(size_t)e.w + t] = xch[set][par][1][0][row] + xch[set][par][1][1][row];
                         }
                     }
-                    if (first_thread) FU_TRACE(2 + set, n_mine, 3);
                     ++n_mine;
                 }
             }
@@ -1207,9 +1222,6 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     // ---------------------------------------------------------------------- teardown
     tc_fence_before();
     __syncthreads();
-#ifdef SABLOCK_TRACE
-    if (blockIdx.x == 0 && threadIdx.x < 8) g_trace[0][5][100 + threadIdx.x][0] = (long long)g_spin[threadIdx.x];
-#endif
     if (sh.abort_flag) {
         if (threadIdx.x == 0) atomicOr(fa.status, kStatTimeout);
         long long t0 = clock64();

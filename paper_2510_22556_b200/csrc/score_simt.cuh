@@ -21,6 +21,19 @@ struct ScoreBufs {
     int n_chunks;
 };
 
+// Single-sweep mode: the caller knows ln sum_j exp(logit_j) of every window row (the prefill's
+// attention kernel keeps it).  Converts it to the log2 units the score kernels work in, once as it
+// is and once negated (the persistent kernel adds it).
+__global__ void lse_import_kernel(const float* __restrict__ row_lse, float* __restrict__ lse2,
+                                  float* __restrict__ neg_lse2, size_t n)
+{
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const float v = row_lse[i] * 1.4426950408889634f;
+    lse2[i] = v;
+    neg_lse2[i] = -v;
+}
+
 template <typename T>
 __global__ void __launch_bounds__(kSimtThreads)
 score_p1_simt(Geo g, const T* __restrict__ q, const T* __restrict__ k, long long ks_tok, long long ks_head,

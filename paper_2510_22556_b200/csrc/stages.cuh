@@ -522,27 +522,136 @@ search_kernel(Geo g, Cands cands, const float* __restrict__ s_ref, const int* __
     }
 }
 
-// Same search for one long segment per CTA; block scores and ranks live in global scratch
-// indexed by absolute token position (disjoint between segments).
-constexpr int kLongThreads = 256;
+// Same search for one long segment per CTA.  A prompt with few delimiters can be one segment of
+// the whole compressible region, so nothing here is quadratic in the segment: Algorithm 2's greedy
+// fill takes blocks in descending (Phi, then lower index) order and stops at the first one that
+// does not fit, and since all blocks but the last have g tokens, where it stops (r*) follows from
+// the rank of the short last block alone.  The retained blocks are then the r* best ones, found
+// by a radix select of the (r* + 1)-th block on the order-preserving integer image of the double
+// block scores (ties to the lower index), which also names the block that is truncated.  Block
+// scores live in global scratch indexed by absolute token position (disjoint between segments).
+constexpr int kLongThreads = 1024;
 
-__device__ __forceinline__ double block_sum_double(double v, double* red)
+__device__ __forceinline__ unsigned long long order_key64(double f)
+{
+    unsigned long long u = (unsigned long long)__double_as_longlong(f);
+    return (u >> 63) ? ~u : (u | 0x8000000000000000ull);
+}
+
+struct LongShared {
+    double red[kLongThreads / 32];
+    int hist[256];
+    int scan[kLongThreads / 32];
+    int b, k, digit, mp;
+};
+
+__device__ __forceinline__ double block_sum_double(double v, LongShared& sm)
 {
     const int tid = threadIdx.x;
     v = warp_sum(v);
-    if ((tid & 31) == 0) red[tid >> 5] = v;
+    if ((tid & 31) == 0) sm.red[tid >> 5] = v;
     __syncthreads();
     double tot = 0.0;
 #pragma unroll
-    for (int w = 0; w < kLongThreads / 32; ++w) tot += red[w];
+    for (int w = 0; w < kLongThreads / 32; ++w) tot += sm.red[w];
     __syncthreads();
     return tot;
+}
+
+__device__ __forceinline__ int block_sum_int(int v, LongShared& sm)
+{
+    const int tid = threadIdx.x;
+    v = warp_sum(v);
+    if ((tid & 31) == 0) sm.scan[tid >> 5] = v;
+    __syncthreads();
+    int tot = 0;
+#pragma unroll
+    for (int w = 0; w < kLongThreads / 32; ++w) tot += sm.scan[w];
+    __syncthreads();
+    return tot;
+}
+
+// The k-th (1-based) of phi[0..nb) in descending order, ties to the lower index: its key and its
+// index.  Block m then ranks before it iff key(m) > thr, or key(m) == thr and m < mp.  Called by
+// every thread of the CTA.
+__device__ __forceinline__ void long_select(const double* __restrict__ phi, int nb, int k, LongShared& sm,
+                                            unsigned long long& thr, int& mp)
+{
+    const int tid = threadIdx.x, lane = tid & 31;
+    unsigned long long prefix = 0, mask = 0;
+    for (int pass = 0; pass < 8; ++pass) {
+        const int shift = 56 - 8 * pass;
+        if (tid < 256) sm.hist[tid] = 0;
+        __syncthreads();
+        for (int m0 = 0; m0 < nb; m0 += kLongThreads) {
+            const int m = m0 + tid;
+            int bin = 256;
+            if (m < nb) {
+                const unsigned long long u = order_key64(phi[m]);
+                if ((u & mask) == prefix) bin = (int)((u >> shift) & 255);
+            }
+            if (__any_sync(0xffffffffu, bin < 256)) {          // one shared-memory atomic per distinct digit per warp
+                const unsigned peers = __match_any_sync(0xffffffffu, bin);
+                if (bin < 256 && lane == __ffs(peers) - 1) atomicAdd(&sm.hist[bin], __popc(peers));
+            }
+        }
+        __syncthreads();
+        if (tid < 32) {
+            // lane l looks at digits 255 - 8 l ... 248 - 8 l, highest first
+            int c[8], mine = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) { c[i] = sm.hist[255 - (8 * lane + i)]; mine += c[i]; }
+            int incl = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += v;
+            }
+            int above = incl - mine;
+            if (above < k && k <= incl) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    if (above + c[i] >= k) { sm.digit = 255 - (8 * lane + i); sm.k = k - above; break; }
+                    above += c[i];
+                }
+            }
+        }
+        __syncthreads();
+        k = sm.k;
+        prefix |= (unsigned long long)sm.digit << shift;
+        mask |= 0xFFull << shift;
+    }
+    // the k-th block, in index order, among those whose key equals the threshold
+    const int chunk = (nb + kLongThreads - 1) / kLongThreads;
+    const int a = min(tid * chunk, nb), z = min(a + chunk, nb);
+    int c = 0;
+    for (int m = a; m < z; ++m) c += (order_key64(phi[m]) == prefix);
+    int inc = c;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += v;
+    }
+    if (lane == 31) sm.scan[tid >> 5] = inc;
+    __syncthreads();
+    int woff = 0;
+    for (int w = 0; w < (tid >> 5); ++w) woff += sm.scan[w];
+    const int excl = woff + inc - c;
+    if (excl < k && k <= excl + c) {
+        int seen = excl;
+        for (int m = a; m < z; ++m)
+            if (order_key64(phi[m]) == prefix && ++seen == k) { sm.mp = m; break; }
+    }
+    __syncthreads();
+    thr = prefix;
+    mp = sm.mp;
+    __syncthreads();
 }
 
 __global__ void __launch_bounds__(kLongThreads)
 search_long_kernel(Geo g, Cands cands, const float* __restrict__ s_ref, const int* __restrict__ seg_start,
                    const unsigned* __restrict__ sel_thr, const int* __restrict__ sel_cut, float tau,
-                   SearchOut out, double* __restrict__ phi_ws, int* __restrict__ rank_ws)
+                   SearchOut out, double* __restrict__ phi_ws)
 {
     const int p = blockIdx.y, layer = p / g.n_seqs, seq = p % g.n_seqs;
     if (geo_identity(g, seq)) return;
@@ -550,95 +659,81 @@ search_long_kernel(Geo g, Cands cands, const float* __restrict__ s_ref, const in
     const size_t off = (size_t)layer * g.total_tokens + g.cu[seq];
     const float* x = s_ref + off;
     const int* sst = seg_start + g.cu[seq] + seq;
-    const unsigned thr = sel_thr[p];
+    const unsigned thr_top = sel_thr[p];
     const int cut = sel_cut[p];
     unsigned* keep = out.keep + (size_t)p * out.keep_words;
     const int tid = threadIdx.x;
-    __shared__ double red[kLongThreads / 32];
-    __shared__ int s_b, s_mp;
+    __shared__ LongShared sm;
 
     for (int li = blockIdx.x; li < count; li += gridDim.x) {
         const int k = out.long_list[(size_t)p * out.long_cap + li];
         const int a = sst[k], z = sst[k + 1], n = z - a;
         const float* sv = x + a;
         double* phi = phi_ws + off + a;
-        int* rank = rank_ws + off + a;
-        if (tid == 0) s_b = 0;
-        __syncthreads();
         int bl = 0;
         double base = 0.0;
         for (int i = tid; i < n; i += kLongThreads) {
-            float v = sv[i];
-            if (in_topb(v, a + i, thr, cut)) { ++bl; base += (double)v; }
+            const float v = sv[i];
+            if (in_topb(v, a + i, thr_top, cut)) { ++bl; base += (double)v; }
         }
-        bl = warp_sum(bl);
-        if ((tid & 31) == 0 && bl) atomicAdd(&s_b, bl);
-        base = block_sum_double(base, red);
-        const int b = s_b;
+        const int b = block_sum_int(bl, sm);
+        base = block_sum_double(base, sm);
         const int lim = min(n, b);
         int g_acc = 1;
         for (int ci = cands.n - 1; ci >= 0; --ci) {
             const int gs = cands.g[ci];
             if (gs > lim) continue;
-            if (gs == 1) {
+            if (gs == 1) {                         // T_k(1) = T_topB within the segment; R_k(1) = 1
                 for (int i = tid; i < n; i += kLongThreads)
-                    if (in_topb(sv[i], a + i, thr, cut)) atomicOr(&keep[(a + i) >> 5], 1u << ((a + i) & 31));
+                    if (in_topb(sv[i], a + i, thr_top, cut)) atomicOr(&keep[(a + i) >> 5], 1u << ((a + i) & 31));
                 g_acc = 1;
                 break;
             }
             const int nb = (n + gs - 1) / gs;
             const int rem = n - (nb - 1) * gs;
-            for (int m = tid; m < nb; m += kLongThreads) {
-                int t0 = m * gs, t1 = min(t0 + gs, n);
+            for (int m = tid; m < nb; m += kLongThreads) {     // block scores Phi, tokens in index order
+                const int t0 = m * gs, t1 = min(t0 + gs, n);
                 double acc = 0.0;
                 for (int t = t0; t < t1; ++t) acc += (double)sv[t];
                 phi[m] = acc;
             }
             __syncthreads();
-            for (int m = tid; m < nb; m += kLongThreads) {
-                double pm = phi[m];
-                int r = 0;
-                for (int m2 = 0; m2 < nb; ++m2) {
-                    double q = phi[m2];
-                    r += (q > pm) || (q == pm && m2 < m);
-                }
-                rank[m] = r;
+            int rl = nb - 1;                                   // rank of the short last block (only matters if it is short)
+            if (rem != gs) {
+                const double pl = phi[nb - 1];
+                int c = 0;
+                for (int m = tid; m < nb - 1; m += kLongThreads) c += phi[m] >= pl;    // earlier index wins a tie
+                rl = block_sum_int(c, sm);
             }
-            if (tid == 0) s_mp = -1;
-            __syncthreads();
             int r_star, m_take;
-            greedy_cut(nb, gs, rem, rank[nb - 1], b, r_star, m_take);
-            if (m_take > 0)
-                for (int m = tid; m < nb; m += kLongThreads) if (rank[m] == r_star) s_mp = m;
-            __syncthreads();
-            const int mp = s_mp;
-            double score = 0.0;
-            for (int i = tid; i < n; i += kLongThreads) {
-                int m = i / gs;
-                bool take = rank[m] < r_star;
+            greedy_cut(nb, gs, rem, rl, b, r_star, m_take);
+            unsigned long long thr = 0;
+            int mp = -1;                                       // the block that is truncated
+            if (r_star < nb) long_select(phi, nb, r_star + 1, sm, thr, mp);
+            const bool all = r_star >= nb;
+            // Retained tokens: the blocks ranked before r*, and the top m_take tokens of block mp
+            // by (score desc, index asc).
+            auto retained = [&](int i) -> bool {
+                const int m = i / gs;
+                if (all) return true;
                 if (m == mp) {
-                    int t0 = mp * gs, t1 = min(t0 + gs, n);
-                    float vi = sv[i];
+                    if (m_take <= 0) return false;
+                    const int t0 = mp * gs, t1 = min(t0 + gs, n);
+                    const float vi = sv[i];
                     int tr = 0;
                     for (int t = t0; t < t1; ++t) tr += (sv[t] > vi) || (sv[t] == vi && t < i);
-                    take = tr < m_take;
+                    return tr < m_take;
                 }
-                if (take) score += (double)sv[i];
-            }
-            score = block_sum_double(score, red);
-            if (score >= (double)tau * base) {
-                for (int i = tid; i < n; i += kLongThreads) {
-                    int m = i / gs;
-                    bool take = rank[m] < r_star;
-                    if (m == mp) {
-                        int t0 = mp * gs, t1 = min(t0 + gs, n);
-                        float vi = sv[i];
-                        int tr = 0;
-                        for (int t = t0; t < t1; ++t) tr += (sv[t] > vi) || (sv[t] == vi && t < i);
-                        take = tr < m_take;
-                    }
-                    if (take) atomicOr(&keep[(a + i) >> 5], 1u << ((a + i) & 31));
-                }
+                const unsigned long long u = order_key64(phi[m]);
+                return u > thr || (u == thr && m < mp);
+            };
+            double score = 0.0;
+            for (int i = tid; i < n; i += kLongThreads)
+                if (retained(i)) score += (double)sv[i];
+            score = block_sum_double(score, sm);
+            if (score >= (double)tau * base) {                 // R_k(g) >= tau (Eqs. 11, 12)
+                for (int i = tid; i < n; i += kLongThreads)
+                    if (retained(i)) atomicOr(&keep[(a + i) >> 5], 1u << ((a + i) & 31));
                 g_acc = gs;
                 break;
             }

@@ -253,6 +253,20 @@ def test_select_long_segments_and_degenerates():
     assert out_idx.cpu().numpy()[:100].tolist() == r["keep"].tolist() == list(range(100))
 
 
+@pytest.mark.parametrize("quantised", [False, True])
+def test_select_very_long_segments(quantised):
+    """A prompt with few or no delimiters is one segment of the whole compressible region (Sec. 3.1):
+    the search must stay linear in the segment length.  Exact against the oracle, ties included."""
+    # the whole 128K region as one segment, at several budgets (the block scores repeat when quantised)
+    for B_tok, tau in ((992, 0.85), (20000, 0.85), (5001, 0.0), (992, 1.0)):
+        _select_case(131040, 32, np.array([131040]), B_tok, [1, 2, 4, 8, 16, 32], tau, quantised, 11 + B_tok)
+    # a 20000-token segment between short ones, odd candidate sizes (short last blocks)
+    rng = np.random.default_rng(9)
+    lens = np.concatenate([rng.geometric(1 / 20.0, 40), [20000], rng.geometric(1 / 20.0, 40), [777, 600]]).astype(np.int64)
+    _select_case(int(lens.sum()), 8, lens, 3000, [1, 2, 3, 5, 7, 9, 11, 13], 0.85, quantised, 12)
+    _select_case(int(lens.sum()), 8, lens, 9000, [1, 3, 7, 13], 0.6, quantised, 13)
+
+
 # ------------------------------------------------------------------ stage 5
 @pytest.mark.parametrize("dtype,Hkv,D", [(torch.bfloat16, 8, 128), (torch.float32, 1, 64), (torch.bfloat16, 2, 64)])
 def test_compact_bytes(dtype, Hkv, D):

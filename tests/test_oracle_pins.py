@@ -160,6 +160,20 @@ def test_gqa_group_mapping():
     assert np.abs(A[0, 0] - 1.0 / (T + 1)).max() > 1e-3
 
 
+def test_prefill_row_lse_generator_is_the_normaliser_of_eq2():
+    """The input generator of the single-sweep mode against the checker: exp(logit - row_lse) must be
+    the attention weight A[h, w, t] of Eq. 2 (logits retyped here from the stored values)."""
+    cfg = synth.Config("lse", 1, 8, 2, 32, 8, (90,), (32,), (1, 2), "bf16", 5000, 4, 2.0, 9, (), 33)
+    b = synth.make_batch(cfg)
+    lse = synth.prefill_row_lse(b.q_win, b.k, b.cu_seqlens)[0, 0].double().numpy()      # [H, W]
+    q, k = b.q_win[0, 0].double(), b.k[0].double()
+    A = oracle.attention(b.q_win[0, 0], b.k[0], cfg.window)
+    T = 90 - cfg.window
+    for h in range(cfg.n_q_heads):
+        logits = (q[h] @ k[:T, h // 4].t()).numpy() / math.sqrt(cfg.head_dim)            # [W, T]
+        np.testing.assert_allclose(np.exp(logits - lse[h][:, None]), A[h], rtol=2e-5)
+
+
 def test_pooling_against_library():
     g = torch.Generator().manual_seed(2)
     s = torch.rand(57, generator=g, dtype=torch.float64)
