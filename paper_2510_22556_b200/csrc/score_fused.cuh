@@ -211,13 +211,15 @@ constexpr int kStepTagShift = 24;       // (epilogue rings) bits 24-31: which us
 constexpr int kFuRing = 16;
 constexpr int kFuSetRing = 8;
 struct FuSched {
-    int4 ring[kFuRing];      // {flags, first token of the tile, T of the sequence, row offset of the outputs}
-    // The steps of each epilogue set once more, in a ring of its own: a set reads only its own
-    // steps (what it must know about the other set's steps is folded into the flags), and a
-    // record says by its tag whether it has been posted, so one look at the slot is enough.
+    // Every step, for the MMA issuer: one tagged flags word (the issuer needs nothing else; ring
+    // position, K stage and parities follow from the step's number).  The tag in bits 24-31 counts
+    // the uses of the slot and is never 0, so one look at the word says whether step n is posted.
+    int ring[kFuRing];
+    // The steps of each epilogue set once more, in a ring of its own: {flags, first token of the
+    // tile, T of the sequence, row offset of the outputs}.  A set reads only its own steps (what it
+    // must know about the other set's steps is folded into the flags); the flags word is tagged in
+    // the same way and is published after the payload.
     int4 sring[2][kFuSetRing];
-    volatile int count;      // steps posted so far
-    volatile int final_;     // the producer has posted its last step
     volatile int lse_fetched;   // log-sum-exp buffers filled so far (helper warp)
     volatile int pub_done;      // phases whose row sums the helper warp has taken out of shared memory
 };
@@ -347,10 +349,11 @@ __device__ __forceinline__ bool wait_counter(const int* ctr, int target, volatil
 }
 
 
-// The step rings and the small counters of FuSched are handed between threads of the CTA with
-// release stores and acquire loads (CTA scope): a reader that sees a count, a tag or a counter
-// value also sees every shared-memory store the writer made before publishing it, and its own
-// later loads of the record cannot be served from before that point.
+// Hand-over of the step rings and the small counters of FuSched between threads of the CTA.  A
+// word that stands for itself (a tagged flags word, a counter) is written and read relaxed.  Where
+// a reader goes on to read what the writer stored BEFORE that word (the payload of a step, the
+// buffer a counter announces), the writer publishes the word with a release store and the reader
+// puts an acquire fence between seeing the word and reading the rest.
 __device__ __forceinline__ void st_release_cta(const volatile void* p, int v)
 {
     asm volatile("st.release.cta.shared.s32 [%0], %1;" ::"r"(smem_u32((const void*)p)), "r"(v) : "memory");
@@ -361,75 +364,78 @@ __device__ __forceinline__ int ld_acquire_cta(const volatile void* p)
     asm volatile("ld.acquire.cta.shared.s32 %0, [%1];" : "=r"(v) : "r"(smem_u32((const void*)p)) : "memory");
     return v;
 }
-__device__ __forceinline__ int4 ld_shared_v4(uint32_t src)
+__device__ __forceinline__ int ld_relaxed_cta(const volatile void* p)
 {
-    int4 out;
-    asm volatile("ld.volatile.shared.v4.s32 {%0, %1, %2, %3}, [%4];" : "=r"(out.x), "=r"(out.y), "=r"(out.z), "=r"(out.w) : "r"(src) : "memory");
-    return out;
+    int v;
+    asm volatile("ld.relaxed.cta.shared.s32 %0, [%1];" : "=r"(v) : "r"(smem_u32((const void*)p)) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_relaxed_cta(const volatile void* p, int v)
+{
+    asm volatile("st.relaxed.cta.shared.s32 [%0], %1;" ::"r"(smem_u32((const void*)p)), "r"(v) : "memory");
+}
+__device__ __forceinline__ void fence_acquire_cta()
+{
+    asm volatile("fence.acq_rel.cta;" ::: "memory");
 }
 
-__device__ __forceinline__ int sched_count(const FuSched& sc) { return ld_acquire_cta(&sc.count); }
-__device__ __forceinline__ void sched_post(FuSched& sc, int idx, int4 step)
+__device__ __forceinline__ int sched_tag(int idx, int ring_len) { return (((idx / ring_len) & 0x7f) + 1) << kStepTagShift; }
+__device__ __forceinline__ bool sched_posted(int fl, int idx, int ring_len)
 {
-    const uint32_t dst = smem_u32(&sc.ring[idx % kFuRing]);
-    asm volatile("st.volatile.shared.v4.s32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(step.x), "r"(step.y), "r"(step.z), "r"(step.w) : "memory");
-    st_release_cta(&sc.count, idx + 1);       // the record before the count
+    return (fl & (0xff << kStepTagShift)) == sched_tag(idx, ring_len);
 }
-// Waits (bounded) until step `idx` is posted and reads it; false when there is no such step or the
-// wait gave up.
-__device__ __forceinline__ bool sched_get(FuSched& sc, int idx, int4& out, volatile int* abort_flag)
+
+// Main ring (MMA issuer): a single word per step.
+__device__ __forceinline__ void sched_post(FuSched& sc, int idx, int flags)
 {
-    if (sched_count(sc) <= idx) {
-        const long long t0 = clock64();
-        while (sched_count(sc) <= idx) {
-            if (ld_acquire_cta(&sc.final_)) {
-                if (sched_count(sc) <= idx) return false;
-                break;
-            }
-            if (*abort_flag || clock64() - t0 > kWaitLimitCycles) { *abort_flag = 1; return false; }
-        }
+    st_relaxed_cta(&sc.ring[idx % kFuRing], flags | sched_tag(idx, kFuRing));
+}
+__device__ __forceinline__ int sched_peek(FuSched& sc, int idx) { return ld_relaxed_cta(&sc.ring[idx % kFuRing]); }
+// Waits (bounded) until step `idx` is posted and returns its flags; false when the wait gave up.
+__device__ __forceinline__ bool sched_get(FuSched& sc, int idx, int& flags, volatile int* abort_flag)
+{
+    long long t0 = 0;
+    int spins = 0;
+    while (true) {
+        flags = sched_peek(sc, idx);
+        if (sched_posted(flags, idx, kFuRing)) return true;
+        if (spins++ == 0) t0 = clock64();
+        if ((spins & 15) == 0 && (*abort_flag || clock64() - t0 > kWaitLimitCycles)) { *abort_flag = 1; return false; }
     }
-    out = ld_shared_v4(smem_u32(&sc.ring[idx % kFuRing]));
-    return true;
 }
 
 // Posts the k-th step of an epilogue set: payload first, then the tagged flags word (release).
 __device__ __forceinline__ void sched_post_set(FuSched& sc, int set, int k, int4 step)
 {
     const uint32_t dst = smem_u32(&sc.sring[set][k % kFuSetRing]);
-    const int tag = ((k / kFuSetRing) & 0x7f) + 1;
-    asm volatile("st.volatile.shared.s32 [%0], %1;" ::"r"(dst + 4), "r"(step.y) : "memory");
-    asm volatile("st.volatile.shared.v2.s32 [%0], {%1, %2};" ::"r"(dst + 8), "r"(step.z), "r"(step.w) : "memory");
-    st_release_cta(&sc.sring[set][k % kFuSetRing], step.x | (tag << kStepTagShift));
+    asm volatile("st.relaxed.cta.shared.s32 [%0], %1;" ::"r"(dst + 4), "r"(step.y) : "memory");
+    asm volatile("st.relaxed.cta.shared.v2.s32 [%0], {%1, %2};" ::"r"(dst + 8), "r"(step.z), "r"(step.w) : "memory");
+    st_release_cta(&sc.sring[set][k % kFuSetRing], step.x | sched_tag(k, kFuSetRing));
 }
-// The flags word of the k-th step of an epilogue set as it stands (posted or not; acquire), and
-// whether a flags word read that way is the posted k-th step.
+// The flags word of the k-th step of an epilogue set as it stands (posted or not), and whether a
+// flags word read that way is the posted k-th step.
 __device__ __forceinline__ int sched_peek_flags(FuSched& sc, int set, int k)
 {
-    return ld_acquire_cta(&sc.sring[set][k % kFuSetRing]);
+    return ld_relaxed_cta(&sc.sring[set][k % kFuSetRing]);
 }
-__device__ __forceinline__ bool sched_flags_posted(int fl, int k)
-{
-    return ((unsigned)fl >> kStepTagShift) == (unsigned)(((k / kFuSetRing) & 0x7f) + 1);
-}
-// Payload of a step whose flags word has been seen posted.
+__device__ __forceinline__ bool sched_flags_posted(int fl, int k) { return sched_posted(fl, k, kFuSetRing); }
+// Payload (.y, .z, .w) of a step whose flags word has been seen posted: the fence orders the read
+// after that sighting.
 __device__ __forceinline__ void sched_payload(FuSched& sc, int set, int k, int4& out)
 {
-    out = ld_shared_v4(smem_u32(&sc.sring[set][k % kFuSetRing]));
+    fence_acquire_cta();
+    const uint32_t src = smem_u32(&sc.sring[set][k % kFuSetRing]);
+    asm volatile("ld.relaxed.cta.shared.s32 %0, [%1];" : "=r"(out.y) : "r"(src + 4) : "memory");
+    asm volatile("ld.relaxed.cta.shared.v2.s32 {%0, %1}, [%2];" : "=r"(out.z), "=r"(out.w) : "r"(src + 8) : "memory");
 }
-// Reads the k-th step of an epilogue set, waiting (bounded) until it is posted: the flags word is
-// acquired first, so a matching tag means the payload read after it is the one posted with it.
-__device__ __forceinline__ bool sched_get_set(FuSched& sc, int set, int k, int4& out, volatile int* abort_flag)
+// Waits (bounded) until the k-th step of an epilogue set is posted and returns its flags.
+__device__ __forceinline__ bool sched_get_set(FuSched& sc, int set, int k, int& flags, volatile int* abort_flag)
 {
     long long t0 = 0;
     int spins = 0;
     while (true) {
-        const int fl = sched_peek_flags(sc, set, k);
-        if (sched_flags_posted(fl, k)) {
-            sched_payload(sc, set, k, out);
-            out.x = fl;
-            return true;
-        }
+        flags = sched_peek_flags(sc, set, k);
+        if (sched_flags_posted(flags, k)) return true;
         if (spins++ == 0) t0 = clock64();
         if ((spins & 15) == 0 && (*abort_flag || clock64() - t0 > kWaitLimitCycles)) { *abort_flag = 1; return false; }
     }
@@ -678,7 +684,7 @@ __device__ __forceinline__ void fu_produce_single(const CUtensorMap* tmQ, const 
             if (qpar) flags |= kStepQPar;
             const int tok0 = (rank + k * fa.cpp) * kTcTile;
             const int4 rec = make_int4(flags, tok0, cur.Tn, cur.layer * g.total_tokens + cur.tok_base);
-            sched_post(sched, n_steps, rec);
+            sched_post(sched, n_steps, flags);
             {
                 const int eset = n_steps & 1;
                 int ef = (flags & ~(7 << kStepRelShift)) | ((ls | ((int)ls_par << 3)) << kStepLseShift);
@@ -710,7 +716,7 @@ __device__ __forceinline__ void fu_produce_single(const CUtensorMap* tmQ, const 
         ls = ls_n;
         if (ls == 0) ls_par ^= 1u;
     }
-    st_release_cta(&sched.final_, 1);
+    sched_post(sched, n_steps, kStepStop);
     for (int es = 0; es < 2; ++es)
         sched_post_set(sched, es, (n_steps + 1 - es) >> 1, make_int4(kStepStop, 0, 0, 0));
 }
@@ -749,9 +755,8 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         for (int i = 0; i < kFuLseSlots; ++i) mbar_init(smem_u32(&sh.lse_full[i]), 1);
         for (int i = 0; i < 2; ++i) mbar_init(smem_u32(&sh.xu[i]), kFuEpiWarps * 16);
         sh.abort_flag = 0;
-        sched.count = 0;
+        for (int i = 0; i < kFuRing; ++i) sched.ring[i] = 0;
         for (int i = 0; i < 2 * kFuSetRing; ++i) (&sched.sring[0][0])[i] = make_int4(0, 0, 0, 0);
-        sched.final_ = 0;
         sched.lse_fetched = 0;
         sched.pub_done = 0;
         fence_mbar_init();
@@ -799,7 +804,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     b_counted = it.b_ph;
                     ++b_idx;
                 }
-                const FuOp op = it.next(ld_acquire_cta(&sched.lse_fetched) > b_idx);
+                const FuOp op = it.next(ld_relaxed_cta(&sched.lse_fetched) > b_idx);   // a hint: the epilogue waits on the buffer's barrier
                 if (op.kind == kOpStop) break;
                 if (op.kind == kOpPairEnd) {
                     // the query block of a phase whose sweep B ended has seen its last product
@@ -828,7 +833,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 if (ph.qpar) flags |= kStepQPar;
                 const int tok0 = op.tile * kTcTile;
                 const int4 rec = make_int4(flags, tok0, ph.Tn, ph.layer * g.total_tokens + ph.tok_base);
-                sched_post(sched, n_steps, rec);
+                sched_post(sched, n_steps, flags);
                 {
                     const int eset = n_steps & 1;
                     int ef = flags & ~(7 << kStepRelShift);
@@ -883,7 +888,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                                 ph.tok_base + tok0, ph.layer, is_b ? pol_b : pol_a);
                 ++n_steps;
             }
-            st_release_cta(&sched.final_, 1);
+            sched_post(sched, n_steps, kStepStop);
             // the end of each epilogue set's list (also after a wait that gave up: the sets then
             // leave through the abort flag)
             for (int es = 0; es < 2; ++es) {
@@ -913,12 +918,11 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             while (true) {
                 if (have_next) {
                     flags = flags_next;
-                } else {
-                    int4 e;
-                    if (!sched_get(sched, n, e, abort_flag)) break;
-                    flags = e.x;
+                } else if (!sched_get(sched, n, flags, abort_flag)) {
+                    break;
                 }
                 have_next = false;
+                if (flags & kStepStop) break;
                 if (flags & (7 << kStepRelShift)) {
 #pragma unroll
                     for (int i = 0; i < kFuQBufs; ++i)
@@ -938,10 +942,8 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 if (!k_ok && !FU_WAIT(5, mbar_wait(bar_k, kpar, abort_flag))) break;
                 tc_fence_after();
                 // the next step's flags, if it is posted, come in while the products are issued
-                if (sched_count(sched) > n + 1) {
-                    flags_next = ld_shared_v4(smem_u32(&sched.ring[(n + 1) % kFuRing])).x;
-                    have_next = true;
-                }
+                flags_next = sched_peek(sched, n + 1);
+                have_next = sched_posted(flags_next, n + 1, kFuRing);
                 const uint32_t k_lo = k_lo0 + st * kTileLo, q_lo = q_lo0 + b * kTileLo;
                 const bool is_b = (flags & kStepB) != 0;
                 fu_issue_tile(tmem + acc * 128u, is_b ? k_lo : q_lo, is_b ? q_lo : k_lo);   // rows = tokens (B) or window rows (A)
@@ -1103,14 +1105,12 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         // Read ahead during a step's exponentials, so that the latencies do not add up between two
         // steps: the flags of the set's next step, and whether its accumulator is complete already.
         int ahead_flags = 0;
-        bool ahead_tfull = false, have_payload = true;
+        bool ahead_tfull = false;
         while (true) {
             if (sched_flags_posted(ahead_flags, n_mine)) {
                 e.x = ahead_flags;
-                have_payload = false;
             } else {
-                if (!sched_get_set(sched, set, n_mine, e, abort_flag)) break;
-                have_payload = true;
+                if (!sched_get_set(sched, set, n_mine, e.x, abort_flag)) break;
                 ahead_tfull = false;
             }
             const int flags = e.x;
@@ -1128,7 +1128,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     tc_fence_before();
                     mbar_arrive(smem_u32(&sh.tempty[set]));   // logits are in registers
                     if (flags & kStepMask) {
-                        if (!have_payload) sched_payload(sched, set, n_mine, e);
+                        sched_payload(sched, set, n_mine, e);
                         const int tok0 = e.y + half * 64;
                         const int lim = e.z + (row & 31);          // causal: key index <= T + w (Eq. 2)
                         chunk_mask(r0, tok0, lim);
@@ -1206,11 +1206,16 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         }
                         xch[set][par][1][half][row] = ent_h;
                         if (!FU_WAIT(20, group_sync(&sh.pbar[set][q4], n_psync, abort_flag))) break;
-                        if (!have_payload) sched_payload(sched, set, n_mine, e);
+                        sched_payload(sched, set, n_mine, e);
                         const int t = e.y + row;
                         if (half == 0 && t < e.z) {
-                            fa.s_out[(size_t)e.w + t] = tot * inv_H;
-                            fa.e_out[(size_t)e.w + t] = xch[set][par][1][0][row] + xch[set][par][1][1][row];
+                            const unsigned o = (unsigned)e.w + (unsigned)t;            // row of the [layer][token] outputs
+                            if (o < (unsigned)g.n_layers * (unsigned)g.total_tokens) {
+                                fa.s_out[o] = tot * inv_H;
+                                fa.e_out[o] = xch[set][par][1][0][row] + xch[set][par][1][1][row];
+                            } else {
+                                atomicOr(fa.status, kStatInternal);                    // a step record that cannot be right
+                            }
                         }
                     }
                     ++n_mine;
