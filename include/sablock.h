@@ -128,6 +128,18 @@ sablock_status_t sablock_workspace_region(const sablock_params_t *p, long long t
  * word is stored to *raw (host) if not NULL. */
 sablock_status_t sablock_read_status(const void *ws, sablock_stream_t stream, int *raw);
 
+/* The same, with the word that follows the status word: raw2 (host int[2]) receives the status
+ * word and, if a bounded wait ran out, which one gave up first:
+ * code | (CTA index << 8) | (warp index << 20).  Codes 1-29 are waits of the persistent score kernel
+ * (1 query-block buffer free, 2 K stage free, 3 query block loaded, 4 accumulator free, 5 K tile
+ * loaded, 6 row sums of a phase in shared memory, 7 accumulator complete, 8 log-sum-exps fetched,
+ * 9 turn at the exponentials, 11 partial-sum slot free, 12 row sums of all CTAs, 13 merged
+ * log-sum-exps, 20 / 21 exchanges inside the epilogue), 30 the look-back of the segmentation scan,
+ * 31 the CTAs of one problem in the Top-B select.  Every such wait is limited to about a second of
+ * device time; the kernel that gave up returns, the later stages still run on whatever was
+ * produced and stay inside their buffers. */
+sablock_status_t sablock_read_status_detail(const void *ws, sablock_stream_t stream, int *raw2);
+
 /* Stage 1 -- semantic segmentation (Sec. 3.1, "Semantic-Aware Segmentation").
  * A token whose id is in the delimiter set is the last token of its segment.
  *  token_ids dev int32[L]; seg_id dev int32[T] (segment index of each token);

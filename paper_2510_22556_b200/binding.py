@@ -6,6 +6,7 @@ Python or torch; if the library is missing the import of `lib()` fails loudly.
 """
 from __future__ import annotations
 
+import contextlib
 import ctypes as C
 import os
 from typing import Optional, Sequence
@@ -26,7 +27,7 @@ EXPORTS = [
     "sablock_read_status", "sablock_segment", "sablock_score", "sablock_select", "sablock_compact",
     "sablock_compress", "sablock_compress_layers", "sablock_compress_layers_host", "sablock_last_launch_count",
     "sablock_params_sizeof", "sablock_workspace_region", "sablock_profile_enable", "sablock_profile_read",
-    "sablock_profile_stage_name", "sablock_segment_static", "sablock_last_cuda_error",
+    "sablock_profile_stage_name", "sablock_segment_static", "sablock_last_cuda_error", "sablock_read_status_detail",
 ]
 
 
@@ -54,38 +55,57 @@ class SablockError(RuntimeError):
 _lib = None
 
 
+def _load(path: str):
+    """dlopens one build of the library and declares the argument types of its entry points."""
+    if not os.path.exists(path):
+        raise ImportError(f"{path} not found: build it with `python -m paper_2510_22556_b200.build` "
+                          "or __graft_entry__.build()")
+    l = C.CDLL(path)
+    l.sablock_status_string.restype = C.c_char_p
+    l.sablock_last_cuda_error.restype = C.c_char_p
+    l.sablock_params_sizeof.restype = C.c_size_t
+    if l.sablock_params_sizeof() != C.sizeof(Params):
+        raise ImportError("sablock_params_t layout mismatch between the library and the binding")
+    l.sablock_workspace_bytes.restype = C.c_size_t
+    l.sablock_workspace_bytes.argtypes = [C.c_void_p, C.c_longlong, C.c_int, C.c_int, C.c_int]
+    vp, ci, sz = C.c_void_p, C.c_int, C.c_size_t
+    l.sablock_read_status.argtypes = [vp, vp, vp]
+    l.sablock_read_status_detail.argtypes = [vp, vp, vp]
+    l.sablock_workspace_region.argtypes = [vp, C.c_longlong, ci, ci, ci, C.c_char_p, vp, vp]
+    l.sablock_params_default.argtypes = [vp]
+    l.sablock_profile_read.argtypes = [ci, vp, ci]
+    l.sablock_profile_stage_name.restype = C.c_char_p
+    l.sablock_segment.argtypes = [vp, vp, ci, vp, vp, vp, vp, sz, vp]
+    l.sablock_segment_static.argtypes = [vp, vp, ci, vp, vp, vp, vp, vp]
+    l.sablock_score.argtypes = [vp, vp, vp, ci, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    l.sablock_select.argtypes = [vp, vp, ci, vp, vp, ci, vp, ci, vp, vp, vp, vp, sz, vp]
+    l.sablock_compact.argtypes = [vp, vp, vp, ci, vp, ci, vp, vp, vp]
+    l.sablock_compress.argtypes = [vp, vp, vp, vp, vp, ci, ci, vp, ci, vp, vp, vp, vp, vp, sz, vp]
+    l.sablock_compress_layers.argtypes = [vp, ci, ci, vp, vp, vp, vp, vp, ci, vp, ci, vp, vp, vp, vp, vp, sz, vp]
+    l.sablock_compress_layers_host.argtypes = [vp, ci, ci, vp, vp, vp, vp, vp, ci, vp, ci, vp, vp, vp, vp,
+                                               vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    return l
+
+
 def lib():
-    """Loads the CUDA library; raises if it has not been built (there is no fallback)."""
+    """The CUDA library; raises if it has not been built (there is no fallback)."""
     global _lib
     if _lib is None:
-        if not os.path.exists(LIB_PATH):
-            raise ImportError(f"{LIB_PATH} not found: build it with `python -m paper_2510_22556_b200.build` "
-                              "or __graft_entry__.build()")
-        l = C.CDLL(LIB_PATH)
-        l.sablock_status_string.restype = C.c_char_p
-        l.sablock_last_cuda_error.restype = C.c_char_p
-        l.sablock_params_sizeof.restype = C.c_size_t
-        if l.sablock_params_sizeof() != C.sizeof(Params):
-            raise ImportError("sablock_params_t layout mismatch between the library and the binding")
-        l.sablock_workspace_bytes.restype = C.c_size_t
-        l.sablock_workspace_bytes.argtypes = [C.c_void_p, C.c_longlong, C.c_int, C.c_int, C.c_int]
-        vp, ci, sz = C.c_void_p, C.c_int, C.c_size_t
-        l.sablock_read_status.argtypes = [vp, vp, vp]
-        l.sablock_workspace_region.argtypes = [vp, C.c_longlong, ci, ci, ci, C.c_char_p, vp, vp]
-        l.sablock_params_default.argtypes = [vp]
-        l.sablock_profile_read.argtypes = [ci, vp, ci]
-        l.sablock_profile_stage_name.restype = C.c_char_p
-        l.sablock_segment.argtypes = [vp, vp, ci, vp, vp, vp, vp, sz, vp]
-        l.sablock_segment_static.argtypes = [vp, vp, ci, vp, vp, vp, vp, vp]
-        l.sablock_score.argtypes = [vp, vp, vp, ci, vp, vp, vp, vp, vp, vp, vp, sz, vp]
-        l.sablock_select.argtypes = [vp, vp, ci, vp, vp, ci, vp, ci, vp, vp, vp, vp, sz, vp]
-        l.sablock_compact.argtypes = [vp, vp, vp, ci, vp, ci, vp, vp, vp]
-        l.sablock_compress.argtypes = [vp, vp, vp, vp, vp, ci, ci, vp, ci, vp, vp, vp, vp, vp, sz, vp]
-        l.sablock_compress_layers.argtypes = [vp, ci, ci, vp, vp, vp, vp, vp, ci, vp, ci, vp, vp, vp, vp, vp, sz, vp]
-        l.sablock_compress_layers_host.argtypes = [vp, ci, ci, vp, vp, vp, vp, vp, ci, vp, ci, vp, vp, vp, vp,
-                                                   vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
-        _lib = l
+        _lib = _load(LIB_PATH)
     return _lib
+
+
+@contextlib.contextmanager
+def use_library(path: str):
+    """Routes every call of this module through another build of the library (the tests of the
+    give-up paths use one with shortened waits) for the duration of the block."""
+    global _lib
+    saved = _lib
+    _lib = _load(path)
+    try:
+        yield _lib
+    finally:
+        _lib = saved
 
 
 def _ptr(t: Optional[torch.Tensor]):
@@ -155,6 +175,13 @@ def read_status(ws: torch.Tensor) -> int:
     raw = C.c_int(0)
     code = lib().sablock_read_status(_ptr(ws), _stream(), C.addressof(raw))
     return code
+
+
+def read_status_detail(ws: torch.Tensor):
+    """(status code, raw status word, code | CTA << 8 | warp << 20 of the first wait that gave up)."""
+    raw = (C.c_int * 2)()
+    code = lib().sablock_read_status_detail(_ptr(ws), _stream(), C.addressof(raw))
+    return code, int(raw[0]), int(raw[1])
 
 
 def profile_enable(slots: int) -> None:

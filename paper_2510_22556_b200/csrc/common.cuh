@@ -18,6 +18,35 @@ constexpr int kMaxCand = SABLOCK_MAX_CANDIDATES;
 constexpr int kStatTimeout = 1;    // a bounded wait ran out
 constexpr int kStatInternal = 2;   // an internal consistency check failed
 
+// Every wait on another thread, CTA or copy is bounded by this many clock cycles (about one
+// second), after which the waiting kernel records the fact and returns.  A test build shortens it.
+#ifndef SABLOCK_WAIT_LIMIT_CYCLES
+#define SABLOCK_WAIT_LIMIT_CYCLES 2000000000LL
+#endif
+constexpr long long kWaitLimitCycles = SABLOCK_WAIT_LIMIT_CYCLES;
+
+// The first wait of a launch that gave up leaves (code | CTA << 8 | warp << 20) in the word after
+// the status word.  Codes 1-29: waits of the persistent score kernel; 30: look-back of the
+// segmentation scan; 31: CTAs of a problem in the Top-B select.
+constexpr int kGiveupSegment = 30;
+constexpr int kGiveupTopB = 31;
+__device__ __forceinline__ void note_giveup(int* status, int code)
+{
+    atomicCAS(status + 1, 0, code | ((int)blockIdx.x << 8) | ((int)(threadIdx.x >> 5) << 20));
+}
+
+// Test builds only (-DSABLOCK_TEST_HOOKS): a word, set from the host, that makes one producer skip
+// its post so that the waiting side runs into its limit.  bit 0: the second tile of the segmentation
+// scan never publishes its state; bit 1: CTA 0 of every Top-B problem never reports its first
+// histogram; bit 2: CTA 0 of the persistent score kernel never reports its row sums of phase 0.
+// Production builds compile none of this.
+#ifdef SABLOCK_TEST_HOOKS
+__device__ int g_test_hooks;
+#define SAB_HOOK(bit) ((g_test_hooks >> (bit)) & 1)
+#else
+#define SAB_HOOK(bit) 0
+#endif
+
 // Geometry of one call: n_layers x n_seqs problems over packed token rows.
 // Problem p = layer * n_seqs + seq.  Per-token arrays are indexed
 // [layer][cu[seq] + t]; per-sequence arrays (segments) [cu[seq] + t].
@@ -131,9 +160,8 @@ __device__ __forceinline__ void mbar_test_wait2(uint32_t bar_a, uint32_t parity_
     ok_b = b != 0;
 }
 
-// Bounded wait: polls the barrier; gives up after `limit` clock cycles or as soon as another
-// role of the CTA has raised *abort.  Returns false on give-up (and raises *abort itself).
-constexpr long long kWaitLimitCycles = 2000000000LL;   // about one second
+// Bounded wait: polls the barrier; gives up after kWaitLimitCycles or as soon as another role of
+// the CTA has raised *abort.  Returns false on give-up (and raises *abort itself).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag)
 {
     if (mbar_try_wait(bar, parity)) return true;

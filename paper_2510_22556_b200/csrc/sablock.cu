@@ -283,7 +283,8 @@ sablock_status_t run_segment(const Plan& pl, const sablock_params_t* p, const in
     dim3 grid(pl.seg_tiles, pl.geo.n_seqs);
     segment_kernel<<<grid, kSegThreads, 0, stream>>>(pl.geo, token_ids, p->delim_bitmap, p->vocab_size, seg_id,
                                                      seg_start, n_seg, at<unsigned long long>(ws, pl.o_tile_state),
-                                                     at<int>(ws, pl.o_ticket), pl.seg_tiles, at<int>(ws, pl.o_status));
+                                                     at<int>(ws, pl.o_ticket), pl.seg_tiles, at<int>(ws, pl.o_status),
+                                                     at<int>(ws, pl.o_status) + 1);
     return check_launch();
 }
 
@@ -714,6 +715,25 @@ sablock_status_t sablock_read_status(const void* ws, sablock_stream_t stream, in
     return SABLOCK_OK;
 }
 
+sablock_status_t sablock_read_status_detail(const void* ws, sablock_stream_t stream, int* raw2)
+{
+    if (!ws || !raw2) return SABLOCK_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(raw2, ws, 2 * sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return SABLOCK_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return SABLOCK_ERR_CUDA;
+    if (raw2[0] & kStatTimeout) return SABLOCK_ERR_TIMEOUT;
+    if (raw2[0] & kStatInternal) return SABLOCK_ERR_INTERNAL;
+    return SABLOCK_OK;
+}
+
+#ifdef SABLOCK_TEST_HOOKS
+// Test builds only: sets the word that makes one producer withhold its post (see common.cuh).
+int sablock_test_set_hooks(int hooks)
+{
+    return (int)cudaMemcpyToSymbol(sab::g_test_hooks, &hooks, sizeof(int));
+}
+#endif
+
 sablock_status_t sablock_segment(const sablock_params_t* p, const int* token_ids, int L, int* seg_id, int* seg_start,
                                  int* n_seg, void* ws, size_t ws_bytes, sablock_stream_t stream)
 {
@@ -771,7 +791,8 @@ sablock_status_t sablock_segment_static(const sablock_params_t* p, const int* to
     g.H = p->n_q_heads; g.Hkv = p->n_kv_heads; g.D = p->head_dim; g.G = g.H / g.Hkv;
     g.cu[0] = 0; g.cu[1] = L;
     segment_kernel<<<dim3(n_tiles, 1), kSegThreads, 0, st>>>(g, token_ids, p->delim_bitmap, p->vocab_size, seg_id, seg_start,
-                                                             n_seg, scratch, ticket, n_tiles, status ? status : own_status);
+                                                             n_seg, scratch, ticket, n_tiles, status ? status : own_status,
+                                                             nullptr);
     return check_launch();
 }
 
@@ -901,12 +922,27 @@ sablock_status_t sablock_compress_layers_host(const sablock_params_t* p, int n_l
 {
     if (!p || !cu_seqlens || n_seqs < 1 || n_seqs > kMaxSeqs || n_layers < 1) return SABLOCK_ERR_INVALID_ARG;
     if (!h_q_win || !h_k || !h_v || !h_token_ids || !h_out_k || !h_out_v || !h_out_idx || !h_out_n_keep ||
-        !dev_q_win || !dev_k || !dev_v || !dev_token_ids)
+        !dev_q_win || !dev_k || !dev_v || !dev_token_ids || !dev_out_k || !dev_out_v || !dev_out_idx || !dev_out_n_keep)
         return SABLOCK_ERR_INVALID_ARG;
     if (p->k_stride_token || p->k_stride_head || p->k_stride_layer || p->v_stride_token || p->v_stride_head ||
         p->v_stride_layer)
         return SABLOCK_ERR_UNSUPPORTED;            // host staging assumes contiguous tensors
-    SAB_TRY(validate_params(p));
+    // Everything the copies below are sized from is checked first: nothing is enqueued on bad arguments.
+    if (budget <= (p->budget_includes_window ? p->window : 0)) return SABLOCK_ERR_INVALID_ARG;
+    if (cu_seqlens[0] != 0) return SABLOCK_ERR_INVALID_ARG;
+    {
+        int max_L = 0;
+        for (int i = 0; i < n_seqs; ++i) {
+            const int L = cu_seqlens[i + 1] - cu_seqlens[i];
+            if (L < 1) return SABLOCK_ERR_INVALID_ARG;
+            if (L > max_L) max_L = L;
+        }
+        Cands cands;
+        SAB_TRY(check_candidates(block_candidates, n_candidates, &cands));
+        Plan pl;
+        SAB_TRY(make_plan(p, n_layers, n_seqs, cu_seqlens, cu_seqlens[n_seqs], max_L, rows_out(p, budget), &pl));
+        if (!ws || ws_bytes < pl.total) return SABLOCK_ERR_WORKSPACE_TOO_SMALL;
+    }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t es = elem_size(p);
     const size_t total = (size_t)cu_seqlens[n_seqs];

@@ -441,11 +441,6 @@ __device__ __forceinline__ bool sched_get_set(FuSched& sc, int set, int k, int& 
     }
 }
 
-// First wait of the launch that gave up: (code, CTA, warp) goes to the word after the status word.
-__device__ __forceinline__ void note_giveup(int* status, int code)
-{
-    atomicCAS(status + 1, 0, code | ((int)blockIdx.x << 8) | ((int)(threadIdx.x >> 5) << 20));
-}
 #define FU_WAIT(code, expr) ((expr) ? true : (note_giveup(fa.status, code), false))
 
 // One 128 x 128 x 128 product into the accumulator at tensor-memory address `d`: eight
@@ -1006,7 +1001,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 ++n_pub;
                 if (lane == 0) {
                     st_release_cta(&sched.pub_done, n_pub);
-                    atomicAdd(fa.arrive + prob * g.Hkv + j, 1);
+                    if (!(SAB_HOOK(2) && blockIdx.x == 0 && phase == 0)) atomicAdd(fa.arrive + prob * g.Hkv + j, 1);
                 }
             }
             if (rank < R) {

@@ -25,7 +25,7 @@ __device__ __forceinline__ int is_delim(int id, const unsigned* bitmap, int voca
 __global__ void __launch_bounds__(kSegThreads)
 segment_kernel(Geo g, const int* __restrict__ token_ids, const unsigned* __restrict__ bitmap, int vocab,
                int* __restrict__ seg_id, int* __restrict__ seg_start, int* __restrict__ n_seg,
-               unsigned long long* tile_state, int* ticket, int max_tiles, int* status)
+               unsigned long long* tile_state, int* ticket, int max_tiles, int* status, int* giveup)
 {
     const int seq = blockIdx.y;
     const int T = geo_L(g, seq) - g.window;
@@ -79,18 +79,20 @@ segment_kernel(Geo g, const int* __restrict__ token_ids, const unsigned* __restr
 
     if (tid == 0) {
         int prefix = 0;
+        const bool withheld = SAB_HOOK(0) && tile == 1;       // test builds: this tile never publishes
         if (tile == 0) {
             *(volatile unsigned long long*)&state[0] = (2ull << 32) | (unsigned)total;
         } else {
-            *(volatile unsigned long long*)&state[tile] = (1ull << 32) | (unsigned)total;
+            if (!withheld) *(volatile unsigned long long*)&state[tile] = (1ull << 32) | (unsigned)total;
             int j = tile - 1;
-            long long spins = 0;
+            const long long t0 = clock64();
             while (j >= 0) {
                 unsigned long long st = *(volatile unsigned long long*)&state[j];
                 unsigned flag = (unsigned)(st >> 32);
                 if (flag == 0) {
-                    if (++spins > (1ll << 24)) {          // bounded: report and carry on
+                    if (clock64() - t0 > kWaitLimitCycles) {   // bounded: report and carry on
                         atomicOr(status, kStatTimeout);
+                        if (giveup) atomicCAS(giveup, 0, kGiveupSegment | ((int)blockIdx.x << 8));
                         break;
                     }
                     __nanosleep(40);
@@ -100,7 +102,7 @@ segment_kernel(Geo g, const int* __restrict__ token_ids, const unsigned* __restr
                 if (flag == 2) break;
                 --j;
             }
-            *(volatile unsigned long long*)&state[tile] = (2ull << 32) | (unsigned)(prefix + total);
+            if (!withheld) *(volatile unsigned long long*)&state[tile] = (2ull << 32) | (unsigned)(prefix + total);
         }
         s_prefix = prefix;
     }
@@ -231,8 +233,9 @@ __device__ __forceinline__ bool top_wait(const int* ctr, int target, int* status
         int v;
         asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ctr) : "memory");
         if (v >= target) return true;
-        if (clock64() - t0 > 2000000000LL) {
+        if (clock64() - t0 > kWaitLimitCycles) {
             atomicOr(status, kStatTimeout);
+            note_giveup(status, kGiveupTopB);
             return false;
         }
         __nanosleep(100);
@@ -289,7 +292,7 @@ topb_kernel(Geo g, const float* __restrict__ s_ref, unsigned* __restrict__ sel_t
             __threadfence();
             __syncthreads();
             if (tid == 0) {
-                atomicAdd(&sc->arrived[pass], 1);
+                if (!(SAB_HOOK(1) && cta == 0 && pass == 0)) atomicAdd(&sc->arrived[pass], 1);
                 s_ok = top_wait(&sc->arrived[pass], n_cta, status) ? 1 : 0;
             }
             __syncthreads();

@@ -99,6 +99,42 @@ def test_argument_checks(lib):
     assert lib.sablock_status_string(3).decode().startswith("workspace")
 
 
+def test_host_buffer_entry_point_checks_before_copying(lib):
+    """sablock_compress_layers_host sizes its copies from cu_seqlens, the budget and the shapes: all of
+    them, the candidates and every pointer are checked before the first copy is enqueued."""
+    p = _params()
+    fake = C.c_void_p(256)                                # never dereferenced: each call must fail on the host
+    ok_c = (C.c_int * 3)(1, 2, 4)
+    big = 1 << 40
+
+    def call(cu=(0, 4096), budget=256, cand=ok_c, n=3, ws=fake, ws_bytes=big, dev_out=fake, h_in=fake):
+        cu_arr = (C.c_int * len(cu))(*cu)
+        return lib.sablock_compress_layers_host(C.addressof(p), 1, len(cu) - 1, h_in, fake, fake, fake, cu_arr, budget,
+                                                cand, n, fake, fake, fake, fake, fake, fake, fake, fake, dev_out, fake,
+                                                fake, fake, ws, ws_bytes, None)
+
+    assert call(cu=(5, 4096)) == 1                        # cu_seqlens[0] must be 0
+    assert call(cu=(0, 4096, 4096)) == 1                  # an empty sequence
+    assert call(cu=(0, 4096, 100)) == 1                   # a negative length
+    assert call(budget=32) == 1 and call(budget=-7) == 1
+    assert call(cand=(C.c_int * 3)(2, 4, 8)) == 1
+    assert call(n=0) == 1
+    assert call(dev_out=None) == 1                        # device outputs may not be NULL
+    assert call(h_in=None) == 1
+    assert call(ws=None) == 3 and call(ws_bytes=4096) == 3
+    bad = _params(n_q_heads=30)
+    cu_arr = (C.c_int * 2)(0, 4096)
+    assert lib.sablock_compress_layers_host(C.addressof(bad), 1, 1, fake, fake, fake, fake, cu_arr, 256, ok_c, 3, fake,
+                                            fake, fake, fake, fake, fake, fake, fake, fake, fake, fake, fake, fake, big,
+                                            None) == 1
+
+
+def test_read_status_detail_rejects_null(lib):
+    raw = (C.c_int * 2)()
+    assert lib.sablock_read_status_detail(None, None, C.addressof(raw)) == 1
+    assert lib.sablock_read_status_detail(C.c_void_p(256), None, None) == 1
+
+
 def test_binding_fails_loudly_without_library(monkeypatch):
     monkeypatch.setattr(B, "_lib", None)
     monkeypatch.setattr(B, "LIB_PATH", "/nonexistent/libsablock.so")
