@@ -69,6 +69,10 @@ CONFIGS = {
     # 4: ragged batch of 16
     "ragged16": Config("ragged16", 32, 32, 8, 128, 32, _ragged_lengths(4, 16, 4096, 16384), (512,),
                        (1, 2, 4, 8, 16), "bf16", 128256, 16, 2.0, 25, (), 4),
+    # the paper's own settings (Sec. 4.1 and 4.5): observation window n_rcnt = 8, search set
+    # {1, 2, 3, 5, 7, 9, 11, 13} (g_max = 13), its budget range, on the same 32-layer stack at 32K
+    "paper8": Config("paper8", 32, 32, 8, 128, 8, (32768,), (128, 256, 512, 1024, 2048),
+                     (1, 2, 3, 5, 7, 9, 11, 13), "bf16", 128256, 16, 2.0, 25, (0.10, 0.50, 0.90), 5),
 }
 
 

@@ -24,7 +24,7 @@ def _params(cfg, bitmap, **kw):
                          bitmap, cfg.vocab, **kw)
 
 
-def run_batch(cfg, batch, budget, layers_to_check=None, **kw):
+def run_batch(cfg, batch, budget, layers_to_check=None, candidates=None, **kw):
     """Runs sablock_compress_layers on a synth.Batch (already on the GPU) and checks the chosen
     layers of every sequence against the oracle, using the scores the same call left in the
     workspace for the tie-aware part."""
@@ -32,8 +32,9 @@ def run_batch(cfg, batch, budget, layers_to_check=None, **kw):
     cu = batch.cu_seqlens
     total, max_L = cu[-1], max(b - a for a, b in zip(cu[:-1], cu[1:]))
     p = _params(cfg, batch.bitmap, **kw)
+    cands = cfg.candidates if candidates is None else tuple(candidates)
     ws = B.alloc_workspace(p, total, max_L, ns, nl)
-    out = B.compress_layers(p, batch.q_win, batch.k, batch.v, batch.token_ids, cu, budget, cfg.candidates, ws)
+    out = B.compress_layers(p, batch.q_win, batch.k, batch.v, batch.token_ids, cu, budget, cands, ws)
     torch.cuda.synchronize()
     assert B.read_status(ws) == 0
     s = B.workspace_view(p, ws, "s", total, max_L, ns, nl)
@@ -46,7 +47,7 @@ def run_batch(cfg, batch, budget, layers_to_check=None, **kw):
         for i in range(ns):
             a, z = cu[i], cu[i + 1]
             infos.append(check_problem(cfg, batch.q_win[l, i], batch.k[l, a:z], batch.v[l, a:z], batch.token_ids[a:z],
-                                       batch.bitmap, cfg.vocab, budget, cfg.candidates, out.out_k[l, i],
+                                       batch.bitmap, cfg.vocab, budget, cands, out.out_k[l, i],
                                        out.out_v[l, i], out.out_idx[l, i], out.n_keep[l, i].item(),
                                        s_gpu=s[l, a:z], e_gpu=e[l, a:z], sr_gpu=sr[l, a:z], params=oparams))
     return out, infos
@@ -162,6 +163,54 @@ def test_paper_defaults_window8_candidates():
     b = synth.make_batch(cfg, device="cuda")
     run_batch(cfg, b, 96)
     run_batch(cfg, b, 1024)
+
+
+@pytest.mark.parametrize("mode", ["sablock", "token_level", "fixed_block_5", "fixed_block_10", "no_segment_scoring"])
+def test_ablation_presets_against_the_oracle(mode):
+    """The variants of the paper's ablation study (Sec. 4.5, Tables 3 and 4) are parameter settings of the
+    same kernels; each is checked against the oracle run with the same settings."""
+    from paper_2510_22556_b200 import modes
+    cfg = synth.CONFIGS["layer8k"]
+    b = synth.make_batch(cfg, device="cuda", seq_lens=[6000])
+    overrides, cands = modes.ablation_presets(cfg.candidates)[mode]
+    out, infos = run_batch(cfg, b, 512, candidates=cands, **overrides)
+    assert out.n_keep.item() == 512
+    if mode == "token_level":                             # exactly the global Top-B of the refined scores
+        r = oracle.compress(b.q_win[0, 0], b.k[0], b.token_ids, b.bitmap, cfg.vocab, 512, (1,))
+        top = np.sort(np.argsort(-r["s_ref"], kind="stable")[: 512 - cfg.window])
+        if infos[0]["exact_vs_pure_oracle"]:
+            assert out.out_idx[0, 0, : 512 - cfg.window].cpu().numpy().tolist() == top.tolist()
+
+
+def test_paper_settings_config_and_diagnostics():
+    """The paper's own settings as a workload (n_rcnt = 8, search set {1,...,13}; two layers of it here),
+    and the two diagnostics computed from the library's outputs against the same figures from the oracle."""
+    from paper_2510_22556_b200 import diagnostics
+    cfg = synth.CONFIGS["paper8"]
+    b = synth.make_batch(cfg, device="cuda", n_layers=2)
+    for budget in (128, 2048):
+        run_batch(cfg, b, budget)
+    L, W = cfg.seq_lens[0], cfg.window
+    p = _params(cfg, b.bitmap)
+    ws = B.alloc_workspace(p, L, L)
+    seg_id, seg_start, n_seg = B.segment(p, b.token_ids, ws)
+    s, e, sr, _ = B.score(p, b.q_win[0, 0], b.k[0], seg_start, n_seg, ws)
+    out_idx, seg_g, seg_b = B.select(p, sr, L, seg_start, n_seg, 1024, cfg.candidates, ws, want_segments=True)
+    torch.cuda.synchronize()
+    ref_id, ref_start = oracle.segment(b.token_ids, W, b.bitmap, cfg.vocab)
+    T = L - W
+    for g in (5, 7, 10):                                   # share of fixed blocks that straddle a boundary (Sec. 2.3)
+        firsts = np.arange(0, T, g)
+        lasts = np.minimum(firsts + g - 1, T - 1)
+        expect = float((ref_id[firsts] != ref_id[lasts]).mean())
+        assert abs(diagnostics.cross_segment_rate(seg_id[:T], g) - expect) < 1e-12
+        assert 0.0 < expect < 1.0
+    ns = int(n_seg.item())
+    r = oracle.select(sr.cpu().double().numpy(), ref_start, 1024 - W, cfg.candidates, tau=float(np.float32(0.85)))
+    hist = diagnostics.block_size_histogram(seg_g, seg_b, ns, cfg.candidates)
+    act = r["g_star"][r["b_k"] > 0]
+    assert hist == {int(c): int((act == c).sum()) for c in cfg.candidates}
+    assert sum(hist.values()) == int((r["b_k"] > 0).sum())
 
 
 def test_strided_kv_cache():

@@ -415,6 +415,41 @@ def test_compress_is_the_composition_of_its_stages(shape, pool_kernel, pool_mode
     assert full["out_idx"].tolist() == list(range(L))           # budget + W >= L: nothing is evicted
 
 
+def test_ablation_settings_reduce_to_their_definitions():
+    """What the ablation presets mean in the checker (Sec. 4.5): token-level retention is the global
+    Top-B of the refined scores; alpha = 0 switches the segment-guided refinement off (Eq. 8); a fixed
+    block size g with tau = 0 is used by every segment that can hold one block of g tokens."""
+    cfg = synth.Config("abl", 1, 8, 2, 32, 8, (400,), (72,), (1, 2, 4, 8), "bf16", 5000, 4, 2.0, 9, (0.4,), 41)
+    b = synth.make_batch(cfg)
+    q, k, ids, W = b.q_win[0, 0], b.k[0], b.token_ids, cfg.window
+    args = (q, k, ids, b.bitmap, cfg.vocab, 72)
+    tok = oracle.compress(*args, (1,))
+    top = np.sort(np.argsort(-tok["s_ref"], kind="stable")[: 72 - W])
+    assert tok["out_idx"][: 72 - W].tolist() == top.tolist()
+    assert set(tok["g_star"][tok["b_k"] > 0].tolist()) == {1}
+    plain = oracle.compress(*args, cfg.candidates, alpha=0.0)
+    np.testing.assert_array_equal(plain["s_ref"], plain["s"])
+    fixed = oracle.compress(*args, (1, 5), tau=0.0)
+    lens = np.diff(fixed["seg_start"])
+    for g, n, bk in zip(fixed["g_star"], lens, fixed["b_k"]):
+        assert g == (0 if bk == 0 else (5 if min(n, bk) >= 5 else 1))
+
+
+def test_cross_segment_rate_helper_against_brute_force():
+    """The motivation statistic of Sec. 2.3 (share of fixed-size blocks that hold tokens of more than one
+    segment): the reporting helper against a per-block recount of the checker's segment ids."""
+    from paper_2510_22556_b200 import diagnostics
+    vocab, W = 1000, 8
+    ids = synth.make_token_ids(3000, vocab, 12, 4)
+    seg_id, _ = oracle.segment(ids, W, synth.delimiter_bitmap(vocab), vocab)
+    T = len(seg_id)
+    for g in (1, 2, 5, 7, 64):
+        crossing = sum(1 for a in range(0, T, g) if len(set(seg_id[a:a + g].tolist())) > 1)
+        n_blocks = (T + g - 1) // g
+        assert abs(diagnostics.cross_segment_rate(torch.from_numpy(seg_id), g) - crossing / n_blocks) < 1e-12
+    assert diagnostics.cross_segment_rate(torch.from_numpy(seg_id), 1) == 0.0
+
+
 def test_gather_is_byte_exact():
     x = torch.randn(50, 2, 8).to(torch.bfloat16)
     idx = np.array([3, 4, 10, 49], np.int32)
