@@ -179,6 +179,18 @@ def gather(x, idx):
     return out
 
 
+def decode_attention(q, k, v):
+    """Attention of one new query token over a cache: q [H, D]; k, v [n, Hkv, D] -> (out [H, D], lse [H])."""
+    qf, kf, vf = _f32(q), _f32(k), _f32(v)
+    H, D = qf.shape
+    n, Hkv, _ = kf.shape
+    out = np.zeros((H, D), np.float64)
+    lse = np.zeros(H, np.float64)
+    lib().sabo_decode_attention(_p(qf, C.c_float), _p(kf, C.c_float), _p(vf, C.c_float), n, H, Hkv, D,
+                                _p(out, C.c_double), _p(lse, C.c_double))
+    return out, lse
+
+
 def compress(q, k, token_ids, bitmap, vocab: int, budget: int, candidates: Sequence[int],
              alpha: float = 0.9, eta: float = 1.0, eps: float = 1e-6, tau: float = 0.85,
              pool_kernel: int = 1, pool_mode: int = 0, budget_includes_window: int = 1):

@@ -336,6 +336,42 @@ void sabo_gather(const uint8_t *src, long long stride_bytes, long long row_bytes
         memcpy(dst + (size_t)i * row_bytes, src + (size_t)idx[i] * stride_bytes, (size_t)row_bytes);
 }
 
+/* ------------------------------------------------------------------ decoding over a cache */
+/* Attention of ONE new query token over a cache of n entries (Eqs. 1-2 with a single query row;
+ * Sec. 4.4 measures decoding over the compressed cache): for every query head h, with the KV head
+ * of its group,  out[h] = sum_i softmax_i(q[h] . k[i] / sqrt(D)) * v[i].  Every entry is visible to
+ * the new token.  q [H][D]; k, v [n][Hkv][D]; out [H][D]; lse [H] = ln of the normaliser. */
+void sabo_decode_attention(const float *q, const float *k, const float *v, int n, int H, int Hkv, int D,
+                           double *out, double *lse)
+{
+    int G = H / Hkv;
+    double inv = 1.0 / sqrt((double)D);
+    double *logit = (double *)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1));
+    for (int h = 0; h < H; ++h) {
+        int j = h / G;
+        const float *qr = q + (size_t)h * D;
+        for (int d = 0; d < D; ++d) out[(size_t)h * D + d] = 0.0;
+        if (n <= 0) { if (lse) lse[h] = -INFINITY; continue; }
+        for (int i = 0; i < n; ++i) {
+            const float *kr = k + ((size_t)i * Hkv + j) * D;
+            double acc = 0.0;
+            for (int d = 0; d < D; ++d) acc += (double)qr[d] * (double)kr[d];
+            logit[i] = acc * inv;
+        }
+        double mx = logit[0];
+        for (int i = 1; i < n; ++i) if (logit[i] > mx) mx = logit[i];
+        double sum = 0.0;
+        for (int i = 0; i < n; ++i) sum += exp(logit[i] - mx);
+        for (int i = 0; i < n; ++i) {
+            double w = exp(logit[i] - mx) / sum;
+            const float *vr = v + ((size_t)i * Hkv + j) * D;
+            for (int d = 0; d < D; ++d) out[(size_t)h * D + d] += w * (double)vr[d];
+        }
+        if (lse) lse[h] = mx + log(sum);
+    }
+    free(logit);
+}
+
 /* ------------------------------------------------------------------ whole pass */
 /* One (layer, sequence).  Outputs: out_idx[n_keep] (ascending positions in the
  * compressible region, then the W window positions), and optionally the stage results.

@@ -450,6 +450,39 @@ def test_cross_segment_rate_helper_against_brute_force():
     assert diagnostics.cross_segment_rate(torch.from_numpy(seg_id), 1) == 0.0
 
 
+@pytest.mark.parametrize("H,Hkv,D,n", [(8, 2, 32, 50), (4, 4, 16, 1), (32, 8, 128, 300), (6, 1, 8, 17)])
+def test_decode_attention_equals_library_softmax(H, Hkv, D, n):
+    """Decoding over a cache (Sec. 4.4): the checker against torch's float64 softmax and matmul, with the
+    grouped-query mapping written out by repeat_interleave."""
+    g = torch.Generator().manual_seed(n)
+    q = torch.randn(H, D, generator=g) * 1.5
+    k = torch.randn(n, Hkv, D, generator=g)
+    v = torch.randn(n, Hkv, D, generator=g)
+    out, lse = oracle.decode_attention(q, k, v)
+    kk = k.double().permute(1, 0, 2).repeat_interleave(H // Hkv, dim=0)        # [H, n, D]
+    vv = v.double().permute(1, 0, 2).repeat_interleave(H // Hkv, dim=0)
+    logits = torch.einsum("hd,hnd->hn", q.double(), kk) / math.sqrt(D)
+    ref = torch.einsum("hn,hnd->hd", torch.softmax(logits, dim=-1), vv)
+    np.testing.assert_allclose(out, ref.numpy(), rtol=1e-11, atol=1e-14)
+    np.testing.assert_allclose(lse, torch.logsumexp(logits, dim=-1).numpy(), rtol=1e-12)
+
+
+def test_decode_attention_closed_forms():
+    """Identical keys: uniform weights, the output is the mean of the values.  One dominant key: its value."""
+    g = torch.Generator().manual_seed(0)
+    q = torch.randn(4, 16, generator=g)
+    k = torch.randn(1, 2, 16, generator=g).expand(9, 2, 16).contiguous()
+    v = torch.randn(9, 2, 16, generator=g)
+    out, lse = oracle.decode_attention(q, k, v)
+    mean_v = v.double().mean(dim=0)                                            # [Hkv, D]
+    np.testing.assert_allclose(out, mean_v.repeat_interleave(2, dim=0).numpy(), rtol=1e-12)
+    k2 = torch.zeros(5, 1, 16)
+    k2[3, 0] = q[0] * 100.0
+    v2 = torch.randn(5, 1, 16, generator=g)
+    out2, _ = oracle.decode_attention(q[:1], k2, v2)
+    np.testing.assert_allclose(out2[0], v2[3, 0].double().numpy(), rtol=1e-9, atol=1e-12)
+
+
 def test_gather_is_byte_exact():
     x = torch.randn(50, 2, 8).to(torch.bfloat16)
     idx = np.array([3, 4, 10, 49], np.int32)
