@@ -243,6 +243,25 @@ sablock_status_t sablock_compress_layers_host(const sablock_params_t *p, int n_l
                                               int *dev_out_n_keep,
                                               void *ws, size_t ws_bytes, sablock_stream_t stream);
 
+/* Decoding over the compacted cache (Sec. 4.4 measures its latency and memory against the full
+ * cache): the attention of ONE new query token per problem over the rows of a cache, Eqs. 1-2 with
+ * a single query row, grouped-query attention as in the scores:
+ *   out[h] = sum_i softmax_i(q[h] . k[i, kv(h)] / sqrt(D)) * v[i, kv(h)],  every row visible.
+ * n_prob problems (layers x sequences, or one layer at a time as a decoder runs them);
+ *  q dev [n_prob, H, D] (dtype of the parameter block); k_cache, v_cache dev [n_prob, n_rows, Hkv, D]:
+ *  what sablock_compress_layers wrote (n_rows = n_out), or a full cache (n_rows = L); element
+ *  strides from the parameter block's k_/v_stride_token, _head, and _layer (between problems),
+ *  0 = contiguous; n_valid dev int32[n_prob] or NULL: rows of each problem that count (out_n_keep),
+ *  NULL = all n_rows; out dev f32 [n_prob, H, D]; lse dev f32 [n_prob, H] or NULL: natural log of
+ *  the softmax normaliser.  Scratch from ws (sablock_decode_workspace_bytes; returns 0 on invalid
+ *  arguments).  Supported: 1, 2 or 4 query heads per KV head, head_dim * element size of 128, 256
+ *  or 512 bytes.  Accumulation is fp32 in a fixed order (row splits merged in index order). */
+size_t sablock_decode_workspace_bytes(const sablock_params_t *p, int n_prob, int n_rows);
+sablock_status_t sablock_decode_attention(const sablock_params_t *p, int n_prob, const void *q,
+                                          const void *k_cache, const void *v_cache, int n_rows,
+                                          const int *n_valid, float *out, float *lse,
+                                          void *ws, size_t ws_bytes, sablock_stream_t stream);
+
 /* Per-stage timing (optional, for benchmarks).  While enabled, every fused call of this
  * thread records CUDA events on its stream between the stages, into the next of `slots`
  * event sets (round robin; the events are created on first use and kept until exit).

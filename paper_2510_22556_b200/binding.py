@@ -28,6 +28,7 @@ EXPORTS = [
     "sablock_compress", "sablock_compress_layers", "sablock_compress_layers_host", "sablock_last_launch_count",
     "sablock_params_sizeof", "sablock_workspace_region", "sablock_profile_enable", "sablock_profile_read",
     "sablock_profile_stage_name", "sablock_segment_static", "sablock_last_cuda_error", "sablock_read_status_detail",
+    "sablock_decode_workspace_bytes", "sablock_decode_attention",
 ]
 
 
@@ -84,6 +85,9 @@ def _load(path: str):
     l.sablock_compress_layers.argtypes = [vp, ci, ci, vp, vp, vp, vp, vp, ci, vp, ci, vp, vp, vp, vp, vp, sz, vp]
     l.sablock_compress_layers_host.argtypes = [vp, ci, ci, vp, vp, vp, vp, vp, ci, vp, ci, vp, vp, vp, vp,
                                                vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    l.sablock_decode_workspace_bytes.restype = C.c_size_t
+    l.sablock_decode_workspace_bytes.argtypes = [vp, ci, ci]
+    l.sablock_decode_attention.argtypes = [vp, ci, vp, vp, vp, ci, vp, vp, vp, vp, sz, vp]
     return l
 
 
@@ -320,3 +324,23 @@ def compress_layers_host(p: Params, h_q, h_k, h_v, h_ids, cu_seqlens, budget, ca
         _ptr(d_q), _ptr(d_k), _ptr(d_v), _ptr(d_ids), _ptr(d_out.out_k), _ptr(d_out.out_v), _ptr(d_out.out_idx),
         _ptr(d_out.n_keep), _ptr(ws), ws.numel(), _stream()), "sablock_compress_layers_host")
     return h_out
+
+
+def decode_attention(p: Params, q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor,
+                     n_valid: Optional[torch.Tensor] = None, ws: Optional[torch.Tensor] = None,
+                     want_lse: bool = False):
+    """One decode step's attention over a cache.  q [n_prob, H, D]; k_cache, v_cache
+    [n_prob, n_rows, Hkv, D] (contiguous).  Returns out f32 [n_prob, H, D] (and lse [n_prob, H])."""
+    n_prob, H, D = q.shape
+    n_rows = k_cache.shape[1]
+    if ws is None:
+        nb = int(lib().sablock_decode_workspace_bytes(C.addressof(p), n_prob, n_rows))
+        if nb == 0:
+            raise SablockError(2, "sablock_decode_workspace_bytes")
+        ws = torch.empty(nb, dtype=torch.uint8, device=q.device)
+    out = torch.empty(n_prob, H, D, dtype=torch.float32, device=q.device)
+    lse = torch.empty(n_prob, H, dtype=torch.float32, device=q.device) if want_lse else None
+    _check(lib().sablock_decode_attention(C.addressof(p), n_prob, _ptr(q), _ptr(k_cache), _ptr(v_cache), n_rows,
+                                          _ptr(n_valid), _ptr(out), _ptr(lse), _ptr(ws), ws.numel(), _stream()),
+           "sablock_decode_attention")
+    return (out, lse) if want_lse else out

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsablock.so")
 SOURCES = ["sablock.cu"]
-HEADERS = ["common.cuh", "stages.cuh", "score_simt.cuh", "score_tc.cuh", "score_fused.cuh"]
+HEADERS = ["common.cuh", "stages.cuh", "score_simt.cuh", "score_tc.cuh", "score_fused.cuh", "decode.cuh"]
 
 
 def _stale(lib: str = LIB) -> bool:

@@ -11,6 +11,7 @@
 #include "score_simt.cuh"
 #include "score_tc.cuh"
 #include "score_fused.cuh"
+#include "decode.cuh"
 
 using namespace sab;
 
@@ -600,6 +601,37 @@ sablock_status_t run_compact(const Geo& g, int n_prob, const sablock_params_t* p
     return check_launch();
 }
 
+// ---- decoding over a cache: launch plan ----------------------------------------------------
+struct DecodePlan { int n_splits, rows_per_split; size_t bytes; };
+
+sablock_status_t decode_plan(const sablock_params_t* p, int n_prob, int n_rows, DecodePlan* dp)
+{
+    SAB_TRY(validate_params(p));
+    if (n_prob < 1 || n_rows < 1) return SABLOCK_ERR_INVALID_ARG;
+    const int G = p->n_q_heads / p->n_kv_heads;
+    const int row_bytes = p->head_dim * elem_size(p);
+    if ((G != 1 && G != 2 && G != 4) || p->head_dim > kDecMaxD || (row_bytes != 128 && row_bytes != 256 && row_bytes != 512))
+        return SABLOCK_ERR_UNSUPPORTED;
+    int splits = (n_rows + kDecThreads - 1) / kDecThreads;
+    if (splits > kDecMaxSplits) splits = kDecMaxSplits;
+    dp->n_splits = splits;
+    dp->rows_per_split = (n_rows + splits - 1) / splits;
+    dp->bytes = align_up(sizeof(float) * (size_t)n_prob * p->n_q_heads * splits * (p->head_dim + 2));
+    return SABLOCK_OK;
+}
+
+template <typename T>
+sablock_status_t launch_decode(const DecodeArgs& a, int G, dim3 grid, cudaStream_t st)
+{
+    switch (G) {
+        case 1: decode_partial_kernel<T, 1><<<grid, kDecThreads, 0, st>>>(a); break;
+        case 2: decode_partial_kernel<T, 2><<<grid, kDecThreads, 0, st>>>(a); break;
+        case 4: decode_partial_kernel<T, 4><<<grid, kDecThreads, 0, st>>>(a); break;
+        default: return SABLOCK_ERR_UNSUPPORTED;
+    }
+    return check_launch();
+}
+
 int rows_out(const sablock_params_t* p, int budget) { return p->budget_includes_window ? budget : budget + p->window; }
 
 }  // namespace
@@ -910,6 +942,51 @@ sablock_status_t sablock_compress(const sablock_params_t* p, const void* q_win, 
     const int cu[2] = {0, L};
     return sablock_compress_layers(p, 1, 1, q_win, k, v, token_ids, cu, budget, block_candidates, n_candidates, out_k,
                                    out_v, out_idx, out_n_keep, ws, ws_bytes, stream);
+}
+
+// ---- decoding over a cache ---------------------------------------------------------------
+size_t sablock_decode_workspace_bytes(const sablock_params_t* p, int n_prob, int n_rows)
+{
+    DecodePlan dp;
+    return decode_plan(p, n_prob, n_rows, &dp) == SABLOCK_OK ? dp.bytes : 0;
+}
+
+sablock_status_t sablock_decode_attention(const sablock_params_t* p, int n_prob, const void* q, const void* k_cache,
+                                          const void* v_cache, int n_rows, const int* n_valid, float* out, float* lse,
+                                          void* ws, size_t ws_bytes, sablock_stream_t stream)
+{
+    t_launches = 0;
+    if (!p || !q || !k_cache || !v_cache || !out) return SABLOCK_ERR_INVALID_ARG;
+    DecodePlan dp;
+    SAB_TRY(decode_plan(p, n_prob, n_rows, &dp));
+    if (!ws || ws_bytes < dp.bytes) return SABLOCK_ERR_WORKSPACE_TOO_SMALL;
+    const int es = elem_size(p);
+    DecodeArgs a;
+    a.q = q; a.k = k_cache; a.v = v_cache;
+    a.k_head = p->k_stride_head ? p->k_stride_head : p->head_dim;
+    a.k_row = p->k_stride_token ? p->k_stride_token : (long long)p->n_kv_heads * p->head_dim;
+    a.k_prob = p->k_stride_layer ? p->k_stride_layer : (long long)n_rows * a.k_row;
+    a.v_head = p->v_stride_head ? p->v_stride_head : p->head_dim;
+    a.v_row = p->v_stride_token ? p->v_stride_token : (long long)p->n_kv_heads * p->head_dim;
+    a.v_prob = p->v_stride_layer ? p->v_stride_layer : (long long)n_rows * a.v_row;
+    const long long strides[] = {a.k_head, a.k_row, a.k_prob, a.v_head, a.v_row, a.v_prob};
+    for (long long x : strides)
+        if ((x * es) % 16) return SABLOCK_ERR_UNSUPPORTED;
+    if ((reinterpret_cast<uintptr_t>(k_cache) | reinterpret_cast<uintptr_t>(v_cache)) & 15) return SABLOCK_ERR_UNSUPPORTED;
+    a.n_valid = n_valid;
+    a.n_rows = n_rows; a.n_splits = dp.n_splits; a.rows_per_split = dp.rows_per_split;
+    a.H = p->n_q_heads; a.Hkv = p->n_kv_heads; a.D = p->head_dim;
+    a.c2 = (float)(1.4426950408889634 / sqrt((double)p->head_dim));
+    a.part = static_cast<float*>(ws);
+    a.out = out; a.lse = lse;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const dim3 grid(dp.n_splits, p->n_kv_heads, n_prob);
+    const int G = p->n_q_heads / p->n_kv_heads;
+    if (p->dtype == SABLOCK_BF16) SAB_TRY(launch_decode<__nv_bfloat16>(a, G, grid, st));
+    else SAB_TRY(launch_decode<float>(a, G, grid, st));
+    const int mt = (p->head_dim + 31) / 32 * 32;
+    decode_merge_kernel<<<dim3(p->n_q_heads, n_prob), mt, 0, st>>>(a);
+    return check_launch();
 }
 
 sablock_status_t sablock_compress_layers_host(const sablock_params_t* p, int n_layers, int n_seqs, const void* h_q_win,
