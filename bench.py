@@ -260,6 +260,8 @@ def run_ours(args):
         if args.sustained_s > 0:
             result["single_sweep"]["sustained"] = sustained(p1, one["ms_step"])
 
+    if rank == 0 and world == 1 and not args.no_decode:
+        result["decode"] = run_decode(B, cfg, batch, p, out, nl, ns, total, max_L, hbm_peak)
     if rank == 0 and world == 1 and not args.no_e2e:
         result["e2e"] = run_e2e(B, cfg, batch, p, ws, out, budget, args)
     elif rank == 0:
@@ -280,6 +282,54 @@ TRAFFIC_CAPTURES = {
     "two_sweep": None,
     "single_sweep": None,
 }
+
+
+def run_decode(B, cfg, batch, p, out, nl, ns, total, max_L, hbm_peak, steps=20):
+    """The consumer of the pass (Sec. 4.4): one decode step's attention, layer by layer as a decoder
+    runs it, over the compacted cache the timed steps left in `out` and over the full cache, with
+    the cache bytes each has to hold.  Extra information beside the metric, not part of it."""
+    H, D = cfg.n_q_heads, cfg.head_dim
+    g = torch.Generator(device="cuda").manual_seed(1234)
+    q_new = torch.randn(nl, ns, H, D, generator=g, device="cuda").to(batch.k.dtype)
+    ws_full = torch.empty(B.lib().sablock_decode_workspace_bytes(ctypes_addr(p), ns, max_L), dtype=torch.uint8, device="cuda")
+    es = batch.k.element_size()
+    row = cfg.n_kv_heads * D * es
+    cu = batch.cu_seqlens
+
+    def compact_step():
+        for l in range(nl):
+            B.decode_attention(p, q_new[l], out.out_k[l], out.out_v[l], n_valid=out.n_keep[l], ws=ws_full)
+
+    def full_step():
+        for l in range(nl):
+            for i in range(ns):                      # sequences of a packed batch have their own lengths
+                B.decode_attention(p, q_new[l, i:i + 1], batch.k[l:l + 1, cu[i]:cu[i + 1]], batch.v[l:l + 1, cu[i]:cu[i + 1]],
+                                   ws=ws_full)
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / steps
+
+    ms_c, ms_f = timed(compact_step), timed(full_step)
+    kv_full, kv_compact = 2 * nl * total * row, 2 * nl * ns * out.n_out * row
+    return {"what": "attention of one new token over all layers' caches, one launch pair per layer",
+            "compact_ms": round(ms_c, 4), "full_ms": round(ms_f, 4), "speedup": round(ms_f / ms_c, 2),
+            "full_cache_gbs": round(kv_full / (ms_f * 1e-3) / 1e9, 1), "full_cache_frac_of_hbm": round(kv_full / (ms_f * 1e-3) / 1e9 / hbm_peak, 4),
+            "kv_bytes_full": kv_full, "kv_bytes_compact": kv_compact,
+            "kv_reduction": round(1.0 - kv_compact / kv_full, 5), "steps": steps}
+
+
+def ctypes_addr(p):
+    import ctypes
+    return ctypes.addressof(p)
 
 
 def run_e2e(B, cfg, batch, p, ws, out, budget, args):
@@ -402,6 +452,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-decode", action="store_true", help="skip the decode-attention comparison (compacted against full cache)")
     ap.add_argument("--no-single-sweep", action="store_true", help="skip the extra loop in single-sweep mode")
     ap.add_argument("--sustained-s", type=float, default=1.5,
                     help="length of the second, power-capped loop per mode in seconds (0 = skip)")

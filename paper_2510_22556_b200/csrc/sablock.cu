@@ -612,7 +612,13 @@ sablock_status_t decode_plan(const sablock_params_t* p, int n_prob, int n_rows, 
     const int row_bytes = p->head_dim * elem_size(p);
     if ((G != 1 && G != 2 && G != 4) || p->head_dim > kDecMaxD || (row_bytes != 128 && row_bytes != 256 && row_bytes != 512))
         return SABLOCK_ERR_UNSUPPORTED;
+    // Row splits: at least 256 rows each, and no more CTAs than a few waves of the device (two
+    // CTAs per SM are resident): the merge that follows reads one partial result per split.
     int splits = (n_rows + kDecThreads - 1) / kDecThreads;
+    const long long ctas_wanted = 8LL * sm_count();
+    const long long per_split = (long long)p->n_kv_heads * n_prob;
+    const int cap = (int)fmax(1.0, (double)(ctas_wanted / per_split));
+    if (splits > cap) splits = cap;
     if (splits > kDecMaxSplits) splits = kDecMaxSplits;
     dp->n_splits = splits;
     dp->rows_per_split = (n_rows + splits - 1) / splits;
@@ -620,16 +626,39 @@ sablock_status_t decode_plan(const sablock_params_t* p, int n_prob, int n_rows, 
     return SABLOCK_OK;
 }
 
-template <typename T>
-sablock_status_t launch_decode(const DecodeArgs& a, int G, dim3 grid, cudaStream_t st)
+template <typename T, int D>
+sablock_status_t launch_decode_d(const DecodeArgs& a, int G, dim3 grid, cudaStream_t st)
 {
+    void (*kern)(DecodeArgs) = nullptr;
     switch (G) {
-        case 1: decode_partial_kernel<T, 1><<<grid, kDecThreads, 0, st>>>(a); break;
-        case 2: decode_partial_kernel<T, 2><<<grid, kDecThreads, 0, st>>>(a); break;
-        case 4: decode_partial_kernel<T, 4><<<grid, kDecThreads, 0, st>>>(a); break;
+        case 1: kern = decode_partial_kernel<T, 1, D>; break;
+        case 2: kern = decode_partial_kernel<T, 2, D>; break;
+        case 4: kern = decode_partial_kernel<T, 4, D>; break;
         default: return SABLOCK_ERR_UNSUPPORTED;
     }
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecSmemBytes) != cudaSuccess)
+        return note_cuda_error(cudaGetLastError(), "shared memory of the decode kernel");
+    kern<<<grid, kDecThreads, kDecSmemBytes, st>>>(a);
     return check_launch();
+}
+
+// head_dim * element size is 128, 256 or 512 bytes (checked by decode_plan)
+sablock_status_t launch_decode(const DecodeArgs& a, bool bf16, int G, dim3 grid, cudaStream_t st)
+{
+    if (bf16) {
+        switch (a.D) {
+            case 64: return launch_decode_d<__nv_bfloat16, 64>(a, G, grid, st);
+            case 128: return launch_decode_d<__nv_bfloat16, 128>(a, G, grid, st);
+            case 256: return launch_decode_d<__nv_bfloat16, 256>(a, G, grid, st);
+        }
+    } else {
+        switch (a.D) {
+            case 32: return launch_decode_d<float, 32>(a, G, grid, st);
+            case 64: return launch_decode_d<float, 64>(a, G, grid, st);
+            case 128: return launch_decode_d<float, 128>(a, G, grid, st);
+        }
+    }
+    return SABLOCK_ERR_UNSUPPORTED;
 }
 
 int rows_out(const sablock_params_t* p, int budget) { return p->budget_includes_window ? budget : budget + p->window; }
@@ -982,8 +1011,7 @@ sablock_status_t sablock_decode_attention(const sablock_params_t* p, int n_prob,
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const dim3 grid(dp.n_splits, p->n_kv_heads, n_prob);
     const int G = p->n_q_heads / p->n_kv_heads;
-    if (p->dtype == SABLOCK_BF16) SAB_TRY(launch_decode<__nv_bfloat16>(a, G, grid, st));
-    else SAB_TRY(launch_decode<float>(a, G, grid, st));
+    SAB_TRY(launch_decode(a, p->dtype == SABLOCK_BF16, G, grid, st));
     const int mt = (p->head_dim + 31) / 32 * 32;
     decode_merge_kernel<<<dim3(p->n_q_heads, n_prob), mt, 0, st>>>(a);
     return check_launch();
