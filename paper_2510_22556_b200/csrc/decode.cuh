@@ -259,38 +259,51 @@ decode_partial_kernel(DecodeArgs a)
 
 // out[p][h][:] = sum over the splits of acc * 2^(m - M) / sum over the splits of l * 2^(m - M).  The
 // weights go through shared memory so that the loads of the D-wide sums are independent of one
-// another; both sums run in split order in every thread.
-__global__ void __launch_bounds__(kDecMaxD)
+// another; four slices of threads take every fourth split each and are added in slice order, so
+// the summation order is fixed.  blockDim = kDecMergeSlices * dpad, dpad = D rounded up to 32.
+constexpr int kDecMergeSlices = 4;
+
+__global__ void __launch_bounds__(kDecMergeSlices * kDecMaxD)
 decode_merge_kernel(DecodeArgs a)
 {
-    const int h = blockIdx.x, p = blockIdx.y, d = threadIdx.x;
+    const int h = blockIdx.x, p = blockIdx.y, tid = threadIdx.x;
     const int D = a.D, ns = a.n_splits;
+    const int dpad = blockDim.x / kDecMergeSlices, slice = tid / dpad, d = tid - slice * dpad;
     const float* base = a.part + ((size_t)p * a.H + h) * ns * (D + 2);
     __shared__ float w_s[kDecMaxSplits], lw_s[kDecMaxSplits];
-    __shared__ float red[kDecMaxD / 32];
+    __shared__ float red[kDecMergeSlices * kDecMaxD / 32];
+    __shared__ float num_s[kDecMergeSlices][kDecMaxD];
     float mx = -INFINITY;
-    for (int s = d; s < ns; s += blockDim.x) mx = fmaxf(mx, base[(size_t)s * (D + 2) + D]);
+    for (int s = tid; s < ns; s += blockDim.x) mx = fmaxf(mx, base[(size_t)s * (D + 2) + D]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    if ((d & 31) == 0) red[d >> 5] = mx;
+    if ((tid & 31) == 0) red[tid >> 5] = mx;
     __syncthreads();
     float M = -INFINITY;
     for (int w = 0; w < (int)(blockDim.x >> 5); ++w) M = fmaxf(M, red[w]);
-    for (int s = d; s < ns; s += blockDim.x) {
+    for (int s = tid; s < ns; s += blockDim.x) {
         const float ms = base[(size_t)s * (D + 2) + D];
         const float w = (ms == -INFINITY || M == -INFINITY) ? 0.f : exp2f(ms - M);      // a split without rows weighs nothing
         w_s[s] = w;
         lw_s[s] = base[(size_t)s * (D + 2) + D + 1] * w;
     }
     __syncthreads();
-    float den = 0.f, num = 0.f;
-    for (int s = 0; s < ns; ++s) den += lw_s[s];
+    float num = 0.f;
     if (d < D) {
 #pragma unroll 8
-        for (int s = 0; s < ns; ++s) num = fmaf(base[(size_t)s * (D + 2) + d], w_s[s], num);
-        a.out[((size_t)p * a.H + h) * D + d] = den > 0.f ? num / den : 0.f;
+        for (int s = slice; s < ns; s += kDecMergeSlices) num = fmaf(base[(size_t)s * (D + 2) + d], w_s[s], num);
+        num_s[slice][d] = num;
     }
-    if (a.lse && d == 0) a.lse[(size_t)p * a.H + h] = den > 0.f ? (M + log2f(den)) * 0.6931471805599453f : -INFINITY;
+    __syncthreads();
+    if (slice == 0 && d < D) {
+        float den = 0.f;
+        for (int s = 0; s < ns; ++s) den += lw_s[s];
+        float tot = 0.f;
+#pragma unroll
+        for (int q = 0; q < kDecMergeSlices; ++q) tot += num_s[q][d];
+        a.out[((size_t)p * a.H + h) * D + d] = den > 0.f ? tot / den : 0.f;
+        if (a.lse && d == 0) a.lse[(size_t)p * a.H + h] = den > 0.f ? (M + log2f(den)) * 0.6931471805599453f : -INFINITY;
+    }
 }
 
 }  // namespace sab

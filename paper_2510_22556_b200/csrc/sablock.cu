@@ -612,10 +612,10 @@ sablock_status_t decode_plan(const sablock_params_t* p, int n_prob, int n_rows, 
     const int row_bytes = p->head_dim * elem_size(p);
     if ((G != 1 && G != 2 && G != 4) || p->head_dim > kDecMaxD || (row_bytes != 128 && row_bytes != 256 && row_bytes != 512))
         return SABLOCK_ERR_UNSUPPORTED;
-    // Row splits: at least 256 rows each, and no more CTAs than a few waves of the device (two
-    // CTAs per SM are resident): the merge that follows reads one partial result per split.
+    // Row splits: at least 256 rows each, and no more CTAs than two waves of the device (two CTAs
+    // per SM are resident): the merge that follows reads one partial result per split.
     int splits = (n_rows + kDecThreads - 1) / kDecThreads;
-    const long long ctas_wanted = 8LL * sm_count();
+    const long long ctas_wanted = 4LL * sm_count();
     const long long per_split = (long long)p->n_kv_heads * n_prob;
     const int cap = (int)fmax(1.0, (double)(ctas_wanted / per_split));
     if (splits > cap) splits = cap;
@@ -1012,7 +1012,7 @@ sablock_status_t sablock_decode_attention(const sablock_params_t* p, int n_prob,
     const dim3 grid(dp.n_splits, p->n_kv_heads, n_prob);
     const int G = p->n_q_heads / p->n_kv_heads;
     SAB_TRY(launch_decode(a, p->dtype == SABLOCK_BF16, G, grid, st));
-    const int mt = (p->head_dim + 31) / 32 * 32;
+    const int mt = kDecMergeSlices * ((p->head_dim + 31) / 32 * 32);
     decode_merge_kernel<<<dim3(p->n_q_heads, n_prob), mt, 0, st>>>(a);
     return check_launch();
 }
