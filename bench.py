@@ -353,7 +353,9 @@ def run_e2e(B, cfg, batch, p, ws, out, budget, args):
     for _ in range(steps):
         step()                      # returns after the stream has drained (results are on the host)
     dt = (time.perf_counter() - t0) / steps
-    h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv, hid))
+    # V is pinned: the gather reads the retained rows from it in place (counted below), the rest is copied
+    v_rows = h_out.out_v.numel() * h_out.out_v.element_size()
+    h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hid)) + v_rows
     d2h = sum(t.numel() * t.element_size() for t in (h_out.out_k, h_out.out_v, h_out.out_idx, h_out.n_keep))
     assert int(h_out.n_keep.min()) == out.n_out
     return {"value": round(cu[-1] / dt, 1), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,

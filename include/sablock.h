@@ -81,7 +81,10 @@ typedef struct sablock_params {
     const unsigned *delim_bitmap;  /* dev: bit (id % 32) of word (id / 32) set <=> id delimits  */
     int vocab_size;                /* ids outside [0, vocab_size) never delimit                 */
     int score_impl;                /* sablock_score_impl_t                                      */
-    int reserved0;
+    int debug_sync;                /* diagnostic aid, default 0: non-zero makes sablock_compress_layers
+                                      wait for the stream after every stage, so that a device fault
+                                      is reported (sablock_last_cuda_error) with the stage that
+                                      raised it; it serialises host and device                  */
     /* Optional, dev f32 [n_layers, n_seqs, H, W] (single-problem calls: [H, W]), or NULL.
      * row_lse[h][w] = ln sum_{j <= T+w} exp(q_{h,w} . k_j / sqrt(D)): the log of the softmax
      * normaliser of Eq. 2 for the query at position T + w, over its causal keys, as the prefill's
@@ -100,9 +103,7 @@ const char *sablock_status_string(sablock_status_t st);
 int sablock_version(void);
 /* Text of the most recent CUDA runtime error an entry point of this thread ran into (which call,
  * after how many kernel launches of that entry point, and the runtime's message); "" if none.
- * With SABLOCK_DEBUG_SYNC=1 in the environment sablock_compress_layers waits for the stream after
- * every stage, so that a device fault is reported here with the stage that raised it (diagnostic
- * aid; it serialises host and device). */
+ * See debug_sync in the parameter block for the stage that raised a device fault. */
 const char *sablock_last_cuda_error(void);
 size_t sablock_params_sizeof(void);   /* sizeof(sablock_params_t) as the library was built */
 
@@ -228,11 +229,14 @@ sablock_status_t sablock_compress_layers(const sablock_params_t *p, int n_layers
                                          void *out_k, void *out_v, int *out_idx, int *out_n_keep,
                                          void *ws, size_t ws_bytes, sablock_stream_t stream);
 
-/* Same pass with HOST inputs and outputs (the end-to-end path): copies q_win, k, v and
- * token_ids from host memory into the caller's device staging buffers (dev_*; same shapes
- * as above), runs sablock_compress_layers, copies out_k, out_v, out_idx, out_n_keep back
- * to host memory and waits for `stream`.  Pinned host memory makes the copies asynchronous
- * with respect to each other; pageable memory also works. */
+/* Same pass with HOST inputs and outputs (the end-to-end path): copies q_win, k and token_ids
+ * from host memory into the caller's device staging buffers (dev_*; same shapes as above), runs
+ * sablock_compress_layers, copies out_k, out_v, out_idx, out_n_keep back to host memory and waits
+ * for `stream`.  The pass reads every key but only the retained rows of v: if h_v is page-locked
+ * (pinned) host memory the gather reads those rows from it in place and dev_v is not written;
+ * otherwise v is copied to dev_v first.  Pinned host memory also makes the copies asynchronous
+ * with respect to each other; pageable memory works too.  All arguments are validated before the
+ * first copy is enqueued. */
 sablock_status_t sablock_compress_layers_host(const sablock_params_t *p, int n_layers, int n_seqs,
                                               const void *h_q_win, const void *h_k, const void *h_v,
                                               const int *h_token_ids, const int *cu_seqlens, int budget,

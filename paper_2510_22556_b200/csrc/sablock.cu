@@ -259,12 +259,11 @@ sablock_status_t check_launch()
 }
 #define SAB_TRY(expr) do { sablock_status_t _s = (expr); if (_s != SABLOCK_OK) return _s; } while (0)
 
-// Diagnostic aid: with SABLOCK_DEBUG_SYNC=1 in the environment the pipeline waits for the stream
+// Diagnostic aid: with debug_sync set in the parameter block the pipeline waits for the stream
 // after every stage, so that a device fault is reported with the stage that raised it.
-sablock_status_t debug_sync(const char* stage, cudaStream_t stream)
+sablock_status_t debug_sync(const sablock_params_t* p, const char* stage, cudaStream_t stream)
 {
-    static const bool on = [] { const char* e = getenv("SABLOCK_DEBUG_SYNC"); return e && e[0] == '1'; }();
-    if (!on) return SABLOCK_OK;
+    if (!p->debug_sync) return SABLOCK_OK;
     const cudaError_t err = cudaStreamSynchronize(stream);
     return err == cudaSuccess ? SABLOCK_OK : note_cuda_error(err, stage);
 }
@@ -945,20 +944,20 @@ sablock_status_t sablock_compress_layers(const sablock_params_t* p, int n_layers
     float* s_raw = p->pool_kernel > 1 ? at<float>(ws, pl.o_s_raw) : s;
     SAB_TRY(run_segment(pl, p, token_ids, seg_id, seg_start, n_seg, ws, st));
     prof_mark(0, st);
-    SAB_TRY(debug_sync("stage segment", st));
+    SAB_TRY(debug_sync(p, "stage segment", st));
     SAB_TRY(run_score(pl, p, q_win, k, s_raw, e, ws, st));
     prof_mark(3, st);
-    SAB_TRY(debug_sync("stage score", st));
+    SAB_TRY(debug_sync(p, "stage score", st));
     SAB_TRY(run_refine(pl, p, s_raw, s, e, seg_start, n_seg, sr, nullptr, 0, st));
     prof_mark(4, st);
-    SAB_TRY(debug_sync("stage refine", st));
+    SAB_TRY(debug_sync(p, "stage refine", st));
     SAB_TRY(run_select(pl, p, sr, seg_start, n_seg, cands, out_idx, out_n_keep, nullptr, nullptr, 0, ws, st));
     prof_mark(7, st);
-    SAB_TRY(debug_sync("stage select", st));
+    SAB_TRY(debug_sync(p, "stage select", st));
     sablock_status_t rc = run_compact(pl.geo, pl.n_prob, p, k, v, out_idx, out_n_keep, 0, out_k, out_v, st);
     prof_mark(8, st);
     prof_end_call();
-    if (rc == SABLOCK_OK) rc = debug_sync("stage compact", st);
+    if (rc == SABLOCK_OK) rc = debug_sync(p, "stage compact", st);
     return rc;
 }
 
@@ -1056,12 +1055,23 @@ sablock_status_t sablock_compress_layers_host(const sablock_params_t* p, int n_l
     const int n_out = rows_out(p, budget);
     const size_t n_prob = (size_t)n_layers * n_seqs;
     const size_t okv_bytes = n_prob * n_out * p->n_kv_heads * p->head_dim * es;
+    // The pass reads every key but only the retained rows of V.  If h_v is pinned (page-locked,
+    // device-accessible) memory the gather reads those rows from it in place; otherwise V is staged
+    // like the rest.
+    const void* v_src = dev_v;
+    {
+        cudaPointerAttributes attr;
+        if (cudaPointerGetAttributes(&attr, h_v) == cudaSuccess && attr.type == cudaMemoryTypeHost && attr.devicePointer)
+            v_src = attr.devicePointer;
+        else
+            cudaGetLastError();
+    }
     if (cudaMemcpyAsync(dev_token_ids, h_token_ids, total * sizeof(int), cudaMemcpyHostToDevice, st) != cudaSuccess ||
         cudaMemcpyAsync(dev_q_win, h_q_win, q_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
         cudaMemcpyAsync(dev_k, h_k, kv_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-        cudaMemcpyAsync(dev_v, h_v, kv_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        (v_src == dev_v && cudaMemcpyAsync(dev_v, h_v, kv_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess))
         return SABLOCK_ERR_CUDA;
-    SAB_TRY(sablock_compress_layers(p, n_layers, n_seqs, dev_q_win, dev_k, dev_v, dev_token_ids, cu_seqlens, budget,
+    SAB_TRY(sablock_compress_layers(p, n_layers, n_seqs, dev_q_win, dev_k, v_src, dev_token_ids, cu_seqlens, budget,
                                     block_candidates, n_candidates, dev_out_k, dev_out_v, dev_out_idx, dev_out_n_keep,
                                     ws, ws_bytes, stream));
     if (cudaMemcpyAsync(h_out_k, dev_out_k, okv_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess ||

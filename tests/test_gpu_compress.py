@@ -228,7 +228,10 @@ def test_strided_kv_cache():
     assert torch.equal(oi, oi2) and torch.equal(ok, ok2) and torch.equal(ov, ov2)
 
 
-def test_host_buffer_entry_point():
+@pytest.mark.parametrize("pinned_v", [True, False])
+def test_host_buffer_entry_point(pinned_v):
+    """Host inputs and outputs.  With V in pinned memory the gather reads the retained rows from it in
+    place (the device staging buffer for V stays untouched); with pageable V it is staged like K."""
     cfg = synth.CONFIGS["layer8k"]
     b = synth.make_batch(cfg, device="cpu", seq_lens=[2048, 1000], n_layers=2)
     d = synth.make_batch(cfg, device="cpu", seq_lens=[2048, 1000], n_layers=2)
@@ -236,8 +239,10 @@ def test_host_buffer_entry_point():
     total, max_L = b.cu_seqlens[-1], 2048
     ws = B.alloc_workspace(p, total, max_L, 2, 2)
     pin = lambda t: t.pin_memory()
-    hq, hk, hv, hid = pin(b.q_win), pin(b.k), pin(b.v), pin(b.token_ids)
+    hq, hk, hid = pin(b.q_win), pin(b.k), pin(b.token_ids)
+    hv = pin(b.v) if pinned_v else b.v.clone()
     dq, dk, dv, did = (torch.empty_like(t, device="cuda") for t in (hq, hk, hv, hid))
+    dv.zero_()
     h_out = B.LayersOut(p, 2, 2, 128, hk.dtype, pinned_host=True)
     d_out = B.LayersOut(p, 2, 2, 128, hk.dtype)
     B.compress_layers_host(p, hq, hk, hv, hid, b.cu_seqlens, 128, cfg.candidates, h_out, dq, dk, dv, did, d_out, ws)
@@ -246,6 +251,7 @@ def test_host_buffer_entry_point():
     torch.cuda.synchronize()
     assert torch.equal(h_out.out_idx, ref.out_idx.cpu()) and torch.equal(h_out.out_k, ref.out_k.cpu())
     assert torch.equal(h_out.out_v, ref.out_v.cpu()) and h_out.n_keep.tolist() == [[128, 128]] * 2
+    assert bool((dv == 0).all()) == pinned_v              # V was staged on the device only when it had to be
 
 
 @pytest.mark.parametrize("L,budget", [
