@@ -386,12 +386,24 @@ sablock_status_t run_score(const Plan& pl, const sablock_params_t* p, const void
         const int min_cpp = (tiles_max + kFuMaxTilesPerCta - 1) / kFuMaxTilesPerCta;
         const int n_cta = pl.use_fused ? fused_cta_limit() : 0;
         if (pl.use_fused && n_cta >= min_cpp && (long long)g.n_layers * g.total_tokens < 0x7fffffffLL) {
-            int groups = n_cta / min_cpp;
-            if (groups > pl.n_prob) groups = pl.n_prob;
-            int cpp = n_cta / groups;
-            if (cpp > tiles_max) cpp = tiles_max;
+            // A CTA holds at most kFuMaxTilesPerCta token tiles of a problem, so a problem needs a
+            // group of ceil(tiles / 7) CTAs; a group that is larger than that leaves its CTAs with
+            // one or two tiles per (problem, KV head) and the hand-over between phases dominates.
+            // The sequences of the call are therefore sorted into classes by the group size they need
+            // (powers of two up to 64, then whatever the longest needs) and every class gets a launch
+            // of its own.  Sequences that are returned unchanged need no scores.
+            int cls_of[kMaxSeqs], cls_need[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+            for (int i = 0; i < g.n_seqs; ++i) {
+                const int L = g.cu[i + 1] - g.cu[i];
+                cls_of[i] = -1;
+                if (L <= g.n_out) continue;
+                const int need = ((L + kTcTile - 1) / kTcTile + kFuMaxTilesPerCta - 1) / kFuMaxTilesPerCta;
+                int c = 0;
+                while (c < 7 && (1 << c) < need) ++c;               // 1, 2, 4, ..., 64, then the rest
+                cls_of[i] = c;
+                if (need > cls_need[c]) cls_need[c] = need;
+            }
             FusedArgs fa;
-            fa.cpp = cpp; fa.n_groups = groups; fa.n_prob = pl.n_prob;
             fa.c2 = c2; fa.eps = p->eps;
             fa.part = at<float2>(ws, pl.o_fpart);
             fa.lse2 = sb.lse2;
@@ -399,15 +411,32 @@ sablock_status_t run_score(const Plan& pl, const sablock_params_t* p, const void
             fa.arrive = at<int>(ws, pl.o_arrive);
             fa.done = at<int>(ws, pl.o_done);
             fa.s_out = s; fa.e_out = e; fa.status = status;
-            Geo geo = g;
-            void* args[] = {&tmQ, &tmK, &geo, &fa};
-            const cudaError_t err = cudaLaunchCooperativeKernel((const void*)score_fused_tc, dim3(groups * cpp), dim3(kFuThreads),
-                                                                args, kFuSmemBytes, stream);
-            if (err != cudaSuccess) {
-                cudaGetLastError();
-                return note_cuda_error(err, "cooperative launch of the score kernel");
+            for (int c = 0; c < 8; ++c) {
+                if (!cls_need[c]) continue;
+                int n_sel = 0, cls_tiles = 0;
+                for (int i = 0; i < g.n_seqs; ++i)
+                    if (cls_of[i] == c) {
+                        fa.sel[n_sel++] = (unsigned char)i;
+                        const int t = (g.cu[i + 1] - g.cu[i] + kTcTile - 1) / kTcTile;
+                        if (t > cls_tiles) cls_tiles = t;
+                    }
+                fa.n_sel = n_sel;
+                fa.n_prob = g.n_layers * n_sel;
+                int groups = n_cta / cls_need[c];
+                if (groups > fa.n_prob) groups = fa.n_prob;
+                int cpp = n_cta / groups;
+                if (cpp > cls_tiles) cpp = cls_tiles;
+                fa.cpp = cpp; fa.n_groups = groups;
+                Geo geo = g;
+                void* args[] = {&tmQ, &tmK, &geo, &fa};
+                const cudaError_t err = cudaLaunchCooperativeKernel((const void*)score_fused_tc, dim3(groups * cpp),
+                                                                    dim3(kFuThreads), args, kFuSmemBytes, stream);
+                if (err != cudaSuccess) {
+                    cudaGetLastError();
+                    return note_cuda_error(err, "cooperative launch of the score kernel");
+                }
+                ++t_launches;
             }
-            ++t_launches;
             prof_mark(1, stream);
             prof_mark(2, stream);
             return SABLOCK_OK;

@@ -44,7 +44,7 @@ constexpr int kFuAbarCol0 = 256;             // columns [0, 256): two logit accu
 constexpr int kFuTmemCols = 512;
 constexpr int kFuLead = 2;                   // sweep A runs at least this many tiles ahead of sweep B
 constexpr int kFuPartSlots = 4;              // ring of per-phase partial buffers in global memory
-constexpr int kFuLseSlots = 8;               // ring of log-sum-exp buffers in shared memory
+constexpr int kFuLseSlots = 16;              // ring of log-sum-exp buffers in shared memory
 constexpr int kFuMaxCtasDev = 256;           // upper bound on the CTAs of one launch
 constexpr int kFuTileBytes = 2 * kAtomBytes; // 128 rows x 128 bf16
 constexpr int kFuSmemBytes = 1024 + (kFuQBufs + kFuStages) * kFuTileBytes;
@@ -60,7 +60,9 @@ constexpr int kFuSmemBytes = 1024 + (kFuQBufs + kFuStages) * kFuTileBytes;
 struct FusedArgs {
     int cpp;                 // CTAs per group (one group works on one problem at a time)
     int n_groups;
-    int n_prob;
+    int n_prob;              // problems of this launch: n_layers x n_sel, numbered layer * n_sel + k
+    int n_sel;               // sequences this launch works on (a call is split into launches by sequence length,
+    unsigned char sel[kMaxSeqs];   // so that short sequences get small groups): their indices
     float c2;                // log2(e) / sqrt(D)
     float eps;
     float2* part;            // [n_groups][kFuPartSlots][cpp][128] row statistics (m, l)
@@ -73,6 +75,17 @@ struct FusedArgs {
     float* e_out;
     int* status;
 };
+
+// Problem v of a launch -> layer, sequence, and the problem's index in the call (layer * n_seqs + seq).
+struct FuProb { int layer, seq, prob; };
+__device__ __forceinline__ FuProb fu_prob(const FusedArgs& fa, const Geo& g, int v)
+{
+    FuProb r;
+    r.layer = v / fa.n_sel;
+    r.seq = fa.sel[v - r.layer * fa.n_sel];
+    r.prob = r.layer * g.n_seqs + r.seq;
+    return r;
+}
 
 struct FuBarriers {
     uint64_t full[kFuStages];
@@ -94,7 +107,8 @@ enum { kOpA = 0, kOpB = 1, kOpPairEnd = 2, kOpStop = 3 };
 
 // What the producer needs to know about one phase = (problem, KV head).
 struct FuPhase {
-    int prob, j;     // problem index and KV head
+    int vp;          // problem number inside the launch
+    int prob, j;     // problem index in the call and KV head
     int layer;
     int Tn;          // compressible length of the sequence
     int tok_base;    // first packed token row of the sequence
@@ -119,20 +133,21 @@ struct FuOp {
 // comes a little later, which costs L2 hits only while it lasts.
 struct FuIter {
     const Geo& g;
+    const FusedArgs& fa;
     int cpp, n_groups, group, rank;
     int n_phases;            // phases of this group
     int a_ph, ia, b_ph, ib;
     int a_buf, b_buf;        // a_ph % 3 and b_ph % 3 (query-block buffers), kept without divisions
     FuPhase pa;              // phase a_ph
     FuPhase q0, q1;          // phases b_ph and b_ph + 1 where those lie behind sweep A
-    __device__ FuIter(const Geo& geo, const FusedArgs& a) : g(geo), cpp(a.cpp), n_groups(a.n_groups)
+    __device__ FuIter(const Geo& geo, const FusedArgs& a) : g(geo), fa(a), cpp(a.cpp), n_groups(a.n_groups)
     {
         group = blockIdx.x / cpp;
         rank = blockIdx.x % cpp;
         const int my_probs = group < n_groups ? (a.n_prob - group + n_groups - 1) / n_groups : 0;
         n_phases = my_probs * g.Hkv;
         a_ph = ia = b_ph = ib = a_buf = b_buf = 0;
-        pa.prob = group; pa.j = -1; pa.n_a = pa.n_b = 0;
+        pa.vp = group; pa.prob = 0; pa.j = -1; pa.n_a = pa.n_b = 0;
         if (n_phases > 0) load_next();
     }
     __device__ int my_tiles(int n) const { return rank < n ? (n - rank + cpp - 1) / cpp : 0; }
@@ -141,10 +156,12 @@ struct FuIter {
     __device__ void load_next()
     {
         if (pa.j >= 0 && pa.j + 1 < g.Hkv) { ++pa.j; return; }
-        if (pa.j >= 0) pa.prob += n_groups;
+        if (pa.j >= 0) pa.vp += n_groups;
         pa.j = 0;
-        pa.layer = pa.prob / g.n_seqs;
-        const int seq = pa.prob - pa.layer * g.n_seqs;
+        const FuProb m = fu_prob(fa, g, pa.vp);
+        pa.layer = m.layer;
+        pa.prob = m.prob;
+        const int seq = m.seq;
         pa.tok_base = g.cu[seq];
         const int L = g.cu[seq + 1] - pa.tok_base;
         pa.Tn = L - g.window;
@@ -204,8 +221,8 @@ constexpr int kStepQPar = 1 << 11;      // parity of that buffer's load
 constexpr int kStepRelShift = 12;       // bits 12-14: before this step, query-block buffer i has seen its last product
 constexpr int kStepMask = 1 << 15;      // sweep A tile that reaches the causal boundary
 constexpr int kStepNewQ = 1 << 16;      // first step that uses this load of the query block
-constexpr int kStepLseShift = 17;       // (epilogue rings) bits 17-19: log-sum-exp buffer of the phase, bit 20: parity of its fill
-constexpr int kStepStop = 1 << 21;      // (epilogue rings) no further step for this set
+constexpr int kStepLseShift = 17;       // (epilogue rings) bits 17-20: log-sum-exp buffer of the phase, bit 21: parity of its fill
+constexpr int kStepStop = 1 << 22;      // (epilogue rings) no further step for this set
 constexpr int kStepTagShift = 24;       // (epilogue rings) bits 24-31: which use of the ring slot this is (never 0)
 
 constexpr int kFuRing = 16;
@@ -557,17 +574,19 @@ __device__ __forceinline__ void accumulate_head16(float (&accw)[16], const uint3
 // between CTAs: the producer walks the phases = (problem, KV head) in which this CTA has token
 // tiles and posts one sweep-B step per tile.  The query block and the 128 log-sum-exps of a phase
 // are fetched one phase ahead: the former into query-block buffer a % 3 (a counts this CTA's
-// phases with tiles), the latter by a bulk copy into log-sum-exp buffer a % 8.  A log-sum-exp
-// buffer is written again eight of this CTA's phases later; the producer is never more than six
-// steps ahead of the oldest step an epilogue set may still be working on (three K stages, two
-// accumulators, the epilogue hands an accumulator back before it is done with the step), and a
-// phase has at least one step, so that buffer has been read for the last time by then.
+// phases with tiles), the latter by a bulk copy into log-sum-exp buffer a % 16.  How far the
+// producer can be ahead of a reader of such a buffer: when it posts step n it has seen the K stage
+// of step n - 1 free, i.e. the products of step n - 4 complete; those were issued after the
+// epilogue of step n - 6 had handed its accumulator back, which it does BEFORE its exponentials,
+// and the other set may likewise still be inside step n - 7.  With one step per phase (short
+// sequences) that is phase a - 7 while the copy for phase a + 1 is issued: nine buffers apart at
+// most, hence sixteen.
 struct FuSinglePhase {
-    int phase, prob, j, layer, tok_base, Tn, n_b;
+    int phase, vp, prob, j, layer, tok_base, Tn, n_b;
 };
 
-__device__ __forceinline__ void fu_single_advance(FuSinglePhase& c, const Geo& g, int group, int n_groups, int rank, int cpp,
-                                                  int n_phases)
+__device__ __forceinline__ void fu_single_advance(FuSinglePhase& c, const Geo& g, const FusedArgs& fa, int group, int n_groups,
+                                                  int rank, int cpp, int n_phases)
 {
     while (true) {
         ++c.phase;
@@ -575,10 +594,12 @@ __device__ __forceinline__ void fu_single_advance(FuSinglePhase& c, const Geo& g
         if (c.j >= 0 && c.j + 1 < g.Hkv) {             // same problem, next KV head
             ++c.j;
         } else {                                       // next problem of the group: the divisions are paid here
-            c.prob = c.j < 0 ? group : c.prob + n_groups;
+            c.vp = c.j < 0 ? group : c.vp + n_groups;
             c.j = 0;
-            c.layer = c.prob / g.n_seqs;
-            const int seq = c.prob - c.layer * g.n_seqs;
+            const FuProb m = fu_prob(fa, g, c.vp);
+            c.layer = m.layer;
+            c.prob = m.prob;
+            const int seq = m.seq;
             c.tok_base = g.cu[seq];
             const int L = g.cu[seq + 1] - c.tok_base;
             c.Tn = L - g.window;
@@ -600,10 +621,10 @@ __device__ __forceinline__ void fu_produce_single(const CUtensorMap* tmQ, const 
     const int my_probs = group < fa.n_groups ? (fa.n_prob - group + fa.n_groups - 1) / fa.n_groups : 0;
     const int n_phases = my_probs * g.Hkv;
     FuSinglePhase cur;
-    cur.phase = -1; cur.prob = 0; cur.j = -1; cur.layer = 0; cur.tok_base = 0; cur.Tn = 0; cur.n_b = 0;
-    fu_single_advance(cur, g, group, fa.n_groups, rank, fa.cpp, n_phases);
+    cur.phase = -1; cur.vp = 0; cur.prob = 0; cur.j = -1; cur.layer = 0; cur.tok_base = 0; cur.Tn = 0; cur.n_b = 0;
+    fu_single_advance(cur, g, fa, group, fa.n_groups, rank, fa.cpp, n_phases);
     FuSinglePhase nxt = cur;
-    if (cur.phase < n_phases) fu_single_advance(nxt, g, group, fa.n_groups, rank, fa.cpp, n_phases);
+    if (cur.phase < n_phases) fu_single_advance(nxt, g, fa, group, fa.n_groups, rank, fa.cpp, n_phases);
 
     // Loads of this CTA's a-th phase with tiles: query block and log-sum-exps.  The buffers must be free.
     auto issue_phase_loads = [&](const FuSinglePhase& ph, int qb, int ls) {
@@ -653,7 +674,7 @@ __device__ __forceinline__ void fu_produce_single(const CUtensorMap* tmQ, const 
             sched_post(sched, n_steps, flags);
             {
                 const int eset = n_steps & 1;
-                int ef = (flags & ~(7 << kStepRelShift)) | ((ls | ((int)ls_par << 3)) << kStepLseShift);
+                int ef = (flags & ~(7 << kStepRelShift)) | ((ls | ((int)ls_par << 4)) << kStepLseShift);
                 if ((eset ? sb1 : sb0) != a_idx) {
                     if (eset) sb1 = a_idx; else sb0 = a_idx;
                     ef |= kStepLseWait;
@@ -676,7 +697,7 @@ __device__ __forceinline__ void fu_produce_single(const CUtensorMap* tmQ, const 
         }
         pending_rel = 1 << (kStepRelShift + qb);           // this phase's query block has seen its last product
         cur = nxt;
-        if (have_next) fu_single_advance(nxt, g, group, fa.n_groups, rank, fa.cpp, n_phases);
+        if (have_next) fu_single_advance(nxt, g, fa, group, fa.n_groups, rank, fa.cpp, n_phases);
         ++a_idx;
         qb = qb_n;
         ls = ls_n;
@@ -753,12 +774,14 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             FuIter it(g, fa);
             // Query blocks are loaded a phase ahead of their first use: phase p goes to buffer p % 3
             // as soon as that buffer's previous tenant (phase p - 3) has seen its last product.
-            int ql_phase = 0, ql_buf = 0, ql_prob = it.group, ql_j = 0;
+            int ql_phase = 0, ql_buf = 0, ql_vp = it.group, ql_prob = 0, ql_j = 0;      // ql_prob: index in the call of problem ql_vp
             unsigned ql_used = 0, ql_par = 0;                  // per buffer: ever loaded, parity of its load count
             bool ql_tiles = false;
-            {
-                const int seq = ql_prob % g.n_seqs, L = geo_L(g, seq);
-                ql_tiles = it.n_phases > 0 && L > g.n_out && it.rank < (L + kTcTile - 1) / kTcTile;
+            if (it.n_phases > 0) {
+                const FuProb m = fu_prob(fa, g, ql_vp);
+                const int L = geo_L(g, m.seq);
+                ql_prob = m.prob;
+                ql_tiles = L > g.n_out && it.rank < (L + kTcTile - 1) / kTcTile;
             }
             unsigned fq_par = 0;                               // the same parities as the work list sees them
             int q_phase = -1, pending_rel = 0, b_idx = -1, b_counted = -1, n_steps = 0;
@@ -805,7 +828,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     int ef = flags & ~(7 << kStepRelShift);
                     if (prev_last_a) ef |= kStepPrevLastA;
                     if (is_b) {
-                        ef |= ((b_idx % kFuLseSlots) | (((b_idx / kFuLseSlots) & 1) << 3)) << kStepLseShift;
+                        ef |= ((b_idx % kFuLseSlots) | (((b_idx / kFuLseSlots) & 1) << 4)) << kStepLseShift;
                         if ((eset ? sb1 : sb0) != b_idx) {
                             if (eset) sb1 = b_idx; else sb0 = b_idx;
                             ef |= kStepLseWait;
@@ -837,9 +860,11 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     ql_buf = ql_buf == kFuQBufs - 1 ? 0 : ql_buf + 1;
                     if (++ql_j == g.Hkv) {
                         ql_j = 0;
-                        ql_prob += it.n_groups;
+                        ql_vp += it.n_groups;
                         if (ql_phase < it.n_phases) {
-                            const int seq = ql_prob % g.n_seqs, L = geo_L(g, seq);
+                            const FuProb m = fu_prob(fa, g, ql_vp);
+                            const int L = geo_L(g, m.seq);
+                            ql_prob = m.prob;
                             ql_tiles = L > g.n_out && it.rank < (L + kTcTile - 1) / kTcTile;
                         }
                     }
@@ -930,7 +955,8 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         const int n_mergers = min(fa.cpp, R);
         int n_fetch = 0, n_pub = 0;
         for (int phase = 0; phase < n_phases; ++phase) {
-            const int prob = group + (phase / g.Hkv) * fa.n_groups, j = phase % g.Hkv, seq = prob % g.n_seqs;
+            const FuProb pm = fu_prob(fa, g, group + (phase / g.Hkv) * fa.n_groups);
+            const int prob = pm.prob, j = phase % g.Hkv, seq = pm.seq;
             if (geo_identity(g, seq)) continue;
             const int L = geo_L(g, seq);
             const int nt1 = (L + kTcTile - 1) / kTcTile, nt2 = (L - g.window + kTcTile - 1) / kTcTile;
@@ -940,8 +966,8 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 // the slot of the partial ring is free once the phase that used it last is merged
                 if (lane == 0 && phase >= kFuPartSlots) {
                     const int old = phase - kFuPartSlots;
-                    ok = FU_WAIT(11, wait_counter(fa.done + (group + (old / g.Hkv) * fa.n_groups) * g.Hkv + old % g.Hkv, n_mergers,
-                                                  abort_flag, fa.status));
+                    const int old_prob = fu_prob(fa, g, group + (old / g.Hkv) * fa.n_groups).prob;
+                    ok = FU_WAIT(11, wait_counter(fa.done + old_prob * g.Hkv + old % g.Hkv, n_mergers, abort_flag, fa.status));
                 }
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
@@ -1111,9 +1137,9 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 if ((flags & kStepLastA) && !publish()) break;
             } else {
                 {
-                    const int lse_slot = (flags >> kStepLseShift) & 7;
+                    const int lse_slot = (flags >> kStepLseShift) & (kFuLseSlots - 1);
                     if (flags & kStepLseWait) {                    // log-sum-exps of this phase (fetched by warp 18)
-                        if (!FU_WAIT(8, mbar_wait(smem_u32(&sh.lse_full[lse_slot]), (uint32_t)((flags >> (kStepLseShift + 3)) & 1), abort_flag)))
+                        if (!FU_WAIT(8, mbar_wait(smem_u32(&sh.lse_full[lse_slot]), (uint32_t)((flags >> (kStepLseShift + 4)) & 1), abort_flag)))
                             break;
                     }
                     if (!ahead_tfull && !FU_WAIT(7, mbar_wait(smem_u32(&sh.tfull[set]), (uint32_t)(n_mine & 1), abort_flag))) break;

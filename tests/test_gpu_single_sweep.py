@@ -79,6 +79,33 @@ def test_single_sweep_runs_are_bit_identical():
     assert torch.equal(runs[0][0], runs[1][0]) and torch.equal(runs[0][1], runs[1][1])
 
 
+def test_many_short_phases_single_sweep():
+    """Short sequences give every CTA one tile step per (problem, KV head) phase, the case in which the
+    producer runs furthest ahead of the epilogue relative to the per-phase buffers (query blocks,
+    log-sum-exps).  64 layers of eight such sequences, twice: identical runs, two problems against the oracle."""
+    cfg = synth.CONFIGS["ragged16"]
+    lens = [2000, 1900, 2100, 1500, 2048, 1800, 2200, 1700]
+    b = synth.make_batch(cfg, device="cuda", n_layers=64, seq_lens=lens)
+    lse = synth.prefill_row_lse(b.q_win, b.k, b.cu_seqlens)
+    p = _params(cfg, b.bitmap, row_lse=lse)
+    total, max_L = b.cu_seqlens[-1], max(lens)
+    ws = B.alloc_workspace(p, total, max_L, len(lens), 64)
+    out = B.LayersOut(p, 64, len(lens), 128, b.k.dtype)
+    runs = []
+    for _ in range(3):
+        B.compress_layers(p, b.q_win, b.k, b.v, b.token_ids, b.cu_seqlens, 128, cfg.candidates, ws, out)
+        torch.cuda.synchronize()
+        assert B.read_status(ws) == 0
+        runs.append((B.workspace_view(p, ws, "s", total, max_L, len(lens), 64).clone(), out.out_idx.clone()))
+    for r in runs[1:]:
+        assert torch.equal(runs[0][0], r[0]) and torch.equal(runs[0][1], r[1])
+    s = runs[0][0]
+    for (l, i) in ((0, 0), (63, 7), (31, 3)):
+        a, z = b.cu_seqlens[i], b.cu_seqlens[i + 1]
+        _, s_ref, _ = oracle.scores(b.q_win[l, i], b.k[l, a:z], eps=float(np.float32(1e-6)))
+        assert_scores_close(s[l, a:z - cfg.window], s_ref, "s")
+
+
 def test_ragged_and_edge_lengths_single_sweep():
     cfg = synth.CONFIGS["ragged16"]
     lens = [128 * 3 - 1, 128 * 3, 128 * 3 + 33, 100, 1024 + 32, 4096 + 17, 33]
