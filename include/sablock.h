@@ -95,7 +95,16 @@ typedef struct sablock_params {
      * row's attention weights by exp(true - given).  The values of sequences that are returned
      * unchanged are ignored. */
     const float *row_lse;
-    int reserved[6];
+    /* Default 0.  The persistent score kernel in its two-sweep mode lets the sweep that accumulates
+     * the softmax normalisers run ahead while the other waits for another CTA; which of its two
+     * groups of warps then sums which token tile depends on timing, so the normalisers (sums of up
+     * to 131072 fp32 terms) can differ in their last bit from run to run, and the scores with them
+     * by about 1e-7 relative.  Non-zero fixes the order of the tile steps: scores are then identical
+     * bit for bit across runs, at about 17 % more time for the score stage on a 128K-token prompt.
+     * Every other mode and kernel (row_lse given, the two-launch and SIMT kernels, all other stages)
+     * is bit-reproducible as it is. */
+    int reproducible;
+    int reserved[5];
 } sablock_params_t;
 
 void sablock_params_default(sablock_params_t *p);
@@ -135,7 +144,7 @@ sablock_status_t sablock_read_status(const void *ws, sablock_stream_t stream, in
  * (1 query-block buffer free, 2 K stage free, 3 query block loaded, 4 accumulator free, 5 K tile
  * loaded, 6 row sums of a phase in shared memory, 7 accumulator complete, 8 log-sum-exps fetched,
  * 9 turn at the exponentials, 11 partial-sum slot free, 12 row sums of all CTAs, 13 merged
- * log-sum-exps, 20 / 21 exchanges inside the epilogue), 30 the look-back of the segmentation scan,
+ * log-sum-exps, 20 / 21 exchanges inside the epilogue, 22 the other epilogue set's previous step), 30 the look-back of the segmentation scan,
  * 31 the CTAs of one problem in the Top-B select.  Every such wait is limited to about a second of
  * device time; the kernel that gave up returns, the later stages still run on whatever was
  * produced and stay inside their buffers. */

@@ -41,7 +41,7 @@ class Params(C.Structure):
         ("alpha", C.c_float), ("eta", C.c_float), ("eps", C.c_float), ("tau", C.c_float),
         ("pool_kernel", C.c_int), ("pool_mode", C.c_int), ("budget_includes_window", C.c_int),
         ("delim_bitmap", C.c_void_p), ("vocab_size", C.c_int),
-        ("score_impl", C.c_int), ("debug_sync", C.c_int), ("row_lse", C.c_void_p), ("reserved", C.c_int * 6),
+        ("score_impl", C.c_int), ("debug_sync", C.c_int), ("row_lse", C.c_void_p), ("reproducible", C.c_int), ("reserved", C.c_int * 5),
     ]
 
 

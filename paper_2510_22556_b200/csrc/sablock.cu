@@ -408,6 +408,7 @@ sablock_status_t run_score(const Plan& pl, const sablock_params_t* p, const void
             fa.part = at<float2>(ws, pl.o_fpart);
             fa.lse2 = sb.lse2;
             fa.neg_lse2 = have_lse ? neg_lse2 : nullptr;
+            fa.fixed_schedule = p->reproducible ? 1 : 0;
             fa.arrive = at<int>(ws, pl.o_arrive);
             fa.done = at<int>(ws, pl.o_done);
             fa.s_out = s; fa.e_out = e; fa.status = status;

@@ -67,6 +67,7 @@ struct FusedArgs {
     float eps;
     float2* part;            // [n_groups][kFuPartSlots][cpp][128] row statistics (m, l)
     float* lse2;             // [n_prob][Hkv * 128] log2-sum-exp2 per window row
+    int fixed_schedule;      // two sweeps: the order of the tile steps ignores when the log-sum-exps arrive
     const float* neg_lse2;   // single-sweep mode: minus the log2-sum-exp2 of every window row, known beforehand
                              // (same layout as lse2; NULL = two sweeps, the kernel works the normalisers out itself)
     int* arrive;             // [n_prob][Hkv]
@@ -98,6 +99,8 @@ struct FuBarriers {
     uint64_t pub_full[2];    // row sums of a phase are in shared memory (all epilogue threads)
     uint64_t lse_full[kFuLseSlots];
     uint64_t xu[2];          // turn of epilogue set s at the exponentials
+    uint64_t adone[2][2];    // epilogue set s has finished its k-th step (k & 1 picks the barrier), its update of
+                             // the head-summed attention included
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -574,13 +577,14 @@ __device__ __forceinline__ void accumulate_head16(float (&accw)[16], const uint3
 // between CTAs: the producer walks the phases = (problem, KV head) in which this CTA has token
 // tiles and posts one sweep-B step per tile.  The query block and the 128 log-sum-exps of a phase
 // are fetched one phase ahead: the former into query-block buffer a % 3 (a counts this CTA's
-// phases with tiles), the latter by a bulk copy into log-sum-exp buffer a % 16.  How far the
-// producer can be ahead of a reader of such a buffer: when it posts step n it has seen the K stage
-// of step n - 1 free, i.e. the products of step n - 4 complete; those were issued after the
-// epilogue of step n - 6 had handed its accumulator back, which it does BEFORE its exponentials,
-// and the other set may likewise still be inside step n - 7.  With one step per phase (short
-// sequences) that is phase a - 7 while the copy for phase a + 1 is issued: nine buffers apart at
-// most, hence sixteen.
+// phases with tiles), the latter by a bulk copy into log-sum-exp buffer a % 16.  The copy for phase
+// a + 1 is issued together with that phase's query block, i.e. once the query-block buffer of phase
+// a - 2 is free: every product up to that phase's last step is complete then.  With one step per
+// phase (the tightest case) those are the products of step n - 2 when step n is being posted; they
+// were issued after the epilogue of step n - 4 had handed its accumulator back, which it does
+// BEFORE its exponentials, and the other set may likewise still be inside step n - 5.  The oldest
+// buffer that can still be read is therefore that of phase a - 5, six buffers from the one being
+// written; sixteen leave a wide margin.
 struct FuSinglePhase {
     int phase, vp, prob, j, layer, tok_base, Tn, n_b;
 };
@@ -741,6 +745,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         }
         for (int i = 0; i < kFuLseSlots; ++i) mbar_init(smem_u32(&sh.lse_full[i]), 1);
         for (int i = 0; i < 2; ++i) mbar_init(smem_u32(&sh.xu[i]), kFuEpiWarps * 16);
+        for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&sh.adone[i >> 1][i & 1]), kFuEpiWarps * 16);
         sh.abort_flag = 0;
         for (int i = 0; i < kFuRing; ++i) sched.ring[i] = 0;
         for (int i = 0; i < 2 * kFuSetRing; ++i) (&sched.sring[0][0])[i] = make_int4(0, 0, 0, 0);
@@ -793,7 +798,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     b_counted = it.b_ph;
                     ++b_idx;
                 }
-                const FuOp op = it.next(ld_relaxed_cta(&sched.lse_fetched) > b_idx);   // a hint: the epilogue waits on the buffer's barrier
+                const FuOp op = it.next(fa.fixed_schedule != 0 || ld_relaxed_cta(&sched.lse_fetched) > b_idx);   // a hint: the epilogue waits on the buffer's barrier
                 if (op.kind == kOpStop) break;
                 if (op.kind == kOpPairEnd) {
                     // the query block of a phase whose sweep B ended has seen its last product
@@ -1132,6 +1137,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     ahead_flags = sched_peek_flags(sched, set, n_mine + 1);
                     rs.add(r1, c2);
                     ahead_tfull = mbar_test_wait(smem_u32(&sh.tfull[set]), (uint32_t)((n_mine + 1) & 1));
+                    mbar_arrive(smem_u32(&sh.adone[set][n_mine & 1]));      // every step counts, so that the parities below hold
                     ++n_mine;
                 }
                 if ((flags & kStepLastA) && !publish()) break;
@@ -1164,7 +1170,17 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     mbar_arrive(smem_u32(&sh.xu[set ^ 1]));
                     accumulate_head16(accw, v3, lj + 96, c2);
                     ahead_tfull = mbar_test_wait(smem_u32(&sh.tfull[set]), (uint32_t)((n_mine + 1) & 1));
-                    // \bar A of this token tile, summed over the KV heads seen so far
+                    // \bar A of this token tile, summed over the KV heads seen so far.  The step before this
+                    // one belongs to the other set and may have updated the same tile's columns (a CTA with
+                    // one tile per phase alternates the sets on it): wait until that set is through its step.
+                    // Set 0's k-th step follows set 1's (k - 1)-th, set 1's k-th follows set 0's k-th.  A set's
+                    // steps alternate between two barriers, so that the other set being one step ahead
+                    // (it cannot be two) does not make the awaited phase ambiguous.
+                    if (set == 1 || n_mine > 0) {
+                        const int ko = n_mine - (set ^ 1);             // the other set's step that precedes this one
+                        if (!FU_WAIT(22, mbar_wait(smem_u32(&sh.adone[set ^ 1][ko & 1]), (uint32_t)((ko >> 1) & 1), abort_flag))) break;
+                        tc_fence_after();
+                    }
                     const uint32_t abar_addr = lane_addr + (uint32_t)(kFuAbarCol0 + ((flags >> kStepKShift) & 7) * 32 + half * 16);
                     if (!(flags & kStepHead0)) {
                         tmem_ld16_issue(abar_addr, v0);
@@ -1210,6 +1226,7 @@ score_fused_tc(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                             }
                         }
                     }
+                    mbar_arrive(smem_u32(&sh.adone[set][n_mine & 1]));
                     ++n_mine;
                 }
             }

@@ -309,6 +309,30 @@ def test_headline_config_full_size():
         assert torch.equal(out.out_k[l, 0], b.k[l, sel]) and torch.equal(out.out_v[l, 0], b.v[l, sel])
 
 
+def test_reproducible_flag_gives_bit_identical_scores_at_full_length():
+    """Two sweeps over a 128K-token prompt: by default the normalisers may differ in their last bit from
+    run to run (which warps sum which tile of the first sweep depends on timing; about 1e-7 relative in
+    the scores, far inside the tolerance); with `reproducible` set the order is fixed and runs agree bit for
+    bit.  Eight layers, five runs each."""
+    cfg = synth.CONFIGS["headline128k"]
+    b = synth.make_batch(cfg, device="cuda", n_layers=8)
+    L = cfg.seq_lens[0]
+    for flag in (1, 0):
+        p = _params(cfg, b.bitmap, reproducible=flag)
+        ws = B.alloc_workspace(p, L, L, 1, 8)
+        runs = []
+        for _ in range(5):
+            out = B.compress_layers(p, b.q_win, b.k, b.v, b.token_ids, b.cu_seqlens, 1024, cfg.candidates, ws)
+            torch.cuda.synchronize()
+            assert B.read_status(ws) == 0
+            runs.append((B.workspace_view(p, ws, "s", L, L, 1, 8)[:, : L - cfg.window].clone(), out.out_idx.clone()))
+        if flag:
+            assert all(torch.equal(runs[0][0], r[0]) and torch.equal(runs[0][1], r[1]) for r in runs[1:])
+        else:
+            worst = max(((runs[0][0] - r[0]).abs() / runs[0][0].abs().clamp_min(1e-30)).max().item() for r in runs[1:])
+            assert worst < 1e-5
+
+
 def test_ragged16_config_full_size():
     cfg = synth.CONFIGS["ragged16"]
     b = synth.make_batch(cfg, device="cuda")
