@@ -289,9 +289,9 @@ def run_ours(args):
 # tokens because every (layer, KV head) streams its own keys).  A capture is quoted only while
 # the kernel is the one it was taken on: otherwise its entry is None.
 TRAFFIC_CAPTURES = {
-    "two_sweep": {"bytes": 547068672 + 6551040, "token_layers": 2 * 131072,
+    "two_sweep": {"bytes": 546839296 + 6333440, "token_layers": 2 * 131072,
                   "source": "profiles/score_fused_tc_headline128k_2layers.txt (2 layers, scaled by layers x tokens)"},
-    "single_sweep": {"bytes": 537507072 + 4996864, "token_layers": 2 * 131072,
+    "single_sweep": {"bytes": 537501184 + 4266496, "token_layers": 2 * 131072,
                      "source": "profiles/score_fused_tc_single_sweep_headline128k_2layers.txt (2 layers, scaled by layers x tokens)"},
 }
 
