@@ -26,6 +26,14 @@
 // split the tile's 128 token columns, in sweep B the 32 window positions.  Warp 18: hand-over
 // between CTAs (publishes this CTA's row sums, merges its share of the rows of all CTAs, fetches
 // the finished log-sum-exps), so that no epilogue thread ever waits on global memory.
+//
+// Single-sweep mode: when the caller passes the log of every window row's normaliser (the prefill's
+// attention kernel keeps it, Sec. 4.1), sweep A, the hand-over warp and the waits between CTAs drop
+// out: the producer posts sweep-B steps only and brings each phase's 128 log-sum-exps into shared
+// memory with a bulk copy, one phase ahead; MMA issuer and epilogue are the same code.
+//
+// A launch works on the sequences of one length class (FusedArgs::sel): the host starts one launch
+// per class so that a problem's group has about ceil(tiles / 7) CTAs and every CTA several tiles.
 #pragma once
 #include "common.cuh"
 #include "score_simt.cuh"

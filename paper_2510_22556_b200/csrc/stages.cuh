@@ -300,15 +300,33 @@ topb_kernel(Geo g, const float* __restrict__ s_ref, unsigned* __restrict__ sel_t
             if (tid < 256) hist[tid] = __ldcg(&sc->hist[pass][tid]);
             __syncthreads();
         }
-        if (tid == 0) {
-            int above = 0, d = 255;
-            for (; d > 0; --d) {
-                if (above + hist[d] >= k) break;
-                above += hist[d];
+        if (tid < 32) {
+            // the digit that holds the k-th key: lane l looks at digits 255 - 8 l ... 248 - 8 l, highest first
+            int c[8], mine = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) { c[i] = hist[255 - (8 * lane + i)]; mine += c[i]; }
+            int incl = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += v;
             }
-            s_k = k - above;
-            s_neq = hist[d];
-            s_prefix = prefix | ((unsigned)d << shift);
+            int above = incl - mine;
+            const int total = __shfl_sync(0xffffffffu, incl, 31);
+            // fewer than k keys left (only with non-finite scores that do not order): the lowest digit
+            if (lane == 31 && total < k) { s_k = k - (total - c[7]); s_neq = c[7]; s_prefix = prefix; }
+            if (above < k && k <= incl) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    if (above + c[i] >= k) {
+                        s_k = k - above;
+                        s_neq = c[i];
+                        s_prefix = prefix | ((unsigned)(255 - (8 * lane + i)) << shift);
+                        break;
+                    }
+                    above += c[i];
+                }
+            }
         }
         __syncthreads();
         k = s_k;
