@@ -333,8 +333,25 @@ def test_reproducible_flag_gives_bit_identical_scores_at_full_length():
             assert worst < 1e-5
 
 
+def check_invariants_every_layer(cfg, b, out, budget):
+    """Every (layer, sequence) of a packed batch: exactly `budget` rows, ascending positions inside the
+    sequence, the window last, and the compacted rows equal to the input rows at those positions."""
+    W = cfg.window
+    assert (out.n_keep.cpu().numpy() == budget).all()
+    idx = out.out_idx.cpu().numpy()                                   # [layers, seqs, budget]
+    assert (np.diff(idx, axis=2) > 0).all()
+    for i, (a, z) in enumerate(zip(b.cu_seqlens[:-1], b.cu_seqlens[1:])):
+        L = z - a
+        assert (idx[:, i, -W:] == np.arange(L - W, L)[None]).all() and idx[:, i].max() < L
+        sel = torch.from_numpy(idx[:, i]).cuda().long() + a           # packed rows, [layers, budget]
+        for l in range(idx.shape[0]):
+            assert torch.equal(out.out_k[l, i], b.k[l, sel[l]]) and torch.equal(out.out_v[l, i], b.v[l, sel[l]])
+
+
 def test_ragged16_config_full_size():
+    """16 sequences of 4096..16384 tokens x 32 layers in one call: layer 7 of every sequence against the
+    oracle in full, every (layer, sequence) for the invariants."""
     cfg = synth.CONFIGS["ragged16"]
     b = synth.make_batch(cfg, device="cuda")
     out, infos = run_batch(cfg, b, 512, layers_to_check=[7])
-    assert (out.n_keep.cpu().numpy() == 512).all()
+    check_invariants_every_layer(cfg, b, out, 512)

@@ -12,7 +12,7 @@ import synth
 from paper_2510_22556_b200 import binding as B
 from paper_2510_22556_b200 import build as build_lib
 from parity import assert_scores_close
-from test_gpu_compress import run_batch, _params
+from test_gpu_compress import check_invariants_every_layer, run_batch, _params
 
 pytestmark = pytest.mark.gpu
 
@@ -118,7 +118,7 @@ def test_ragged16_config_full_size_single_sweep():
     cfg = synth.CONFIGS["ragged16"]
     b = synth.make_batch(cfg, device="cuda")
     out, infos = _with_lse(cfg, b, 512, layers_to_check=[7])
-    assert (out.n_keep.cpu().numpy() == 512).all()
+    check_invariants_every_layer(cfg, b, out, 512)
 
 
 def test_headline_config_full_size_single_sweep():
